@@ -1,0 +1,152 @@
+/* frog.h -- C ABI of the FROG range-filtering k-ANN search library (CUDA, sm_100a).
+ *
+ * The calls follow the paper's problem statement (Sec. 2.1: objects (v_i, a_i), a query
+ * (v_q, [l_q, r_q], k), L2 distance) and the argument list of its Alg. 2
+ * FROGSearch(ENC, v_q, l_q, r_q, k, ef_s, epn, H, N, B).  All of the search runs in CUDA
+ * kernels; there is no CPU fallback.  Nothing here throws, aborts or traps: every call
+ * returns an int status (0 = FROG_OK) that frog_strerror() turns into text.
+ *
+ * Index file (little-endian): a 256-byte header
+ *     char magic[8]="FROGIDX1"; u32 version=1, d, d_pad, H, m, n_inv, ef_c, patience;
+ *     f32 beta, gamma; u64 n, seed; u32 bot=0xFFFFFFFF, reserved;
+ *     u64 off_sorted_attr, off_rank2id, off_vectors, off_enc, file_bytes;
+ * followed, at 128-byte-aligned offsets, by
+ *     sorted_attr[n]   int32   attribute of the object of rank r, ascending (Sec. 4)
+ *     rank2id[n]       int32   original object id of rank r
+ *     vectors[n*d_pad] fp32    row r = vector of rank r, zero-padded to d_pad = 4*ceil(d/4)
+ *     enc[n*H*m]       uint32  ENC block of rank r: H rows (layer 0 = root) of m ranks,
+ *                              0xFFFFFFFF = empty (the n x H x m array of Sec. 4)
+ */
+#ifndef FROG_H_
+#define FROG_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct frog_index frog_index_t; /* opaque; owns its device and host buffers */
+
+enum {
+    FROG_OK = 0,
+    FROG_ERR_INVALID_ARG = 1,   /* null pointer, k < 1, k > beam_width, beam_width out of range ... */
+    FROG_ERR_IO = 2,            /* file cannot be opened / read */
+    FROG_ERR_FORMAT = 3,        /* magic, version, sizes or offsets inconsistent */
+    FROG_ERR_NOMEM = 4,         /* host or device allocation failed */
+    FROG_ERR_CUDA = 5,          /* a CUDA runtime call failed; see frog_last_cuda_error() */
+    FROG_ERR_UNSUPPORTED = 6    /* parameter combination the kernels do not cover */
+};
+
+/* Limits of the search kernels. */
+#define FROG_MAX_BEAM_WIDTH 512 /* ef_s */
+#define FROG_MAX_BUDGET 32      /* B and epn */
+
+typedef struct {
+    int64_t n;          /* objects */
+    int32_t d;          /* dimensionality of the data */
+    int32_t d_pad;      /* floats per stored row (multiple of 4) */
+    int32_t H;          /* retained layers of the segment tree (Sec. 4) */
+    int32_t m;          /* ENCs per vertex per layer */
+    int32_t n_inv;      /* deepest layers omitted */
+    int32_t ef_c;       /* construction-time pool width */
+    int32_t patience;   /* construction-time early-termination patience */
+    float beta, gamma;  /* fusion-distance parameters (Eq. 3) used at construction */
+    uint64_t seed;
+    int32_t device;     /* CUDA device holding the index */
+    int64_t device_bytes; /* bytes of device memory owned by the index */
+} frog_index_info_t;
+
+/* Optional query-time parameters (Alg. 2 arguments other than k and ef_s). */
+typedef struct {
+    int32_t epn;        /* entry points, 1..32; 0 = default 16 (paper Sec. 8.1.4) */
+    int32_t budget;     /* expansion budget B, 1..32; 0 = default 16 */
+    int32_t max_iters;  /* hard cap on expansions per query; 0 = default 16 * beam_width */
+    int32_t no_hotspot; /* nonzero: scan all H layers instead of the hotspot (ablation) */
+    uint64_t seed;      /* seed of the entry-point generator */
+    int32_t hash_bits;  /* log2 of the per-query visited-table slots; 0 = chosen from beam_width */
+    int32_t reserved;
+} frog_params_t;
+
+/* Per-query status bits written by frog_search_ex. */
+#define FROG_ST_EMPTY 1u     /* lo > hi or no object in [lo, hi]: row is all padding */
+#define FROG_ST_EXACT 2u     /* range holds <= beam_width objects: answered by exact scan */
+#define FROG_ST_ITER_CAP 4u  /* expansion cap hit; the current pool was returned */
+#define FROG_ST_SHORT 8u     /* fewer than k results; tail is padding */
+
+/* frog_index_load: read an index file, copy its four arrays to `device`, return a handle.
+ * (Paper Sec. 8.1.3: index and database stay resident in GPU memory.)  Host pointer in, the
+ * handle is owned by the caller until frog_index_free.  Errors: INVALID_ARG, IO, FORMAT,
+ * NOMEM, CUDA. */
+int frog_index_load(const char* path, int device, frog_index_t** out);
+
+/* frog_index_from_host: the same from arrays already in host memory (layout as in the file;
+ * vectors are n x d_pad).  The arrays are copied; the caller keeps ownership of its own. */
+int frog_index_from_host(const int32_t* sorted_attr, const int32_t* rank2id, const float* vectors,
+                         const uint32_t* enc, const frog_index_info_t* shape, int device,
+                         frog_index_t** out);
+
+/* Release device and host memory of an index (null is allowed).  Synchronises the device. */
+void frog_index_free(frog_index_t* index);
+
+int frog_index_info(const frog_index_t* index, frog_index_info_t* out);
+
+/* frog_search: batched FROGSearch (Alg. 2, with Alg. 3 once per query and Alg. 4 plus the lazy
+ * hash check of Sec. 7.3.2 at every expansion), one query per warp of a persistent kernel.
+ *   queries    DEVICE, nq x d fp32 row-major (d = index dimensionality)
+ *   lo, hi     DEVICE, nq int32, inclusive attribute bounds of each query
+ *   k          results per query, 1 <= k <= beam_width
+ *   beam_width ef_s of Alg. 2, 1..FROG_MAX_BEAM_WIDTH
+ *   out_ids    DEVICE, nq x k int32: ORIGINAL object ids, ascending (distance, rank); -1 padding
+ *   out_dists  DEVICE, nq x k fp32: L2 distances (not squared), ascending; +inf padding
+ *   stream     cudaStream_t (as void*); the call only enqueues work and returns
+ * The caller owns all buffers and keeps them alive until the stream reaches the end of the
+ * call.  Calls on the same index must not overlap on the GPU (they share the index's small
+ * scratch: a work counter); serialise them on one stream or with events.  nq == 0 is a no-op.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA (launch failure).  Per-query conditions (empty range,
+ * iteration cap, fewer than k results) are not errors; see frog_search_ex. */
+int frog_search(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
+                int nq, int k, int beam_width, int32_t* out_ids, float* out_dists, void* stream);
+
+/* frog_search_ex: frog_search with explicit parameters and optional per-query outputs.
+ *   params  HOST, may be null (defaults)
+ *   status  DEVICE nq uint32 or null: FROG_ST_* bits
+ *   stats   DEVICE nq x 4 uint32 or null: {expansions, ENC rows the scan needed, ENs admitted
+ *           by Alg. 4, distance evaluations}
+ *   trace   DEVICE nq x trace_cap uint32 or null: row q = [len, then per expansion
+ *           u, |EN(u)|, EN(u)[0..]] (ranks), records appended until the first that would
+ *           exceed trace_cap-1 words.  Selects a
+ *           slower kernel instantiation; meant for tests. */
+int frog_search_ex(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
+                   int nq, int k, int beam_width, const frog_params_t* params,
+                   int32_t* out_ids, float* out_dists, uint32_t* status, uint32_t* stats,
+                   uint32_t* trace, int trace_cap, void* stream);
+
+/* frog_exact_search: exact filtered kNN (Def. 2 of Sec. 2.1) by scanning the contiguous rank
+ * slab of each query (Sec. 4: an attribute range is a contiguous rank interval), one CTA per
+ * query.  Same buffers and conventions as frog_search; 1 <= k <= FROG_MAX_BEAM_WIDTH.  Used for ground truth
+ * and as the pre-filtering reference. */
+int frog_exact_search(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
+                      int nq, int k, int32_t* out_ids, float* out_dists, void* stream);
+
+/* frog_search_host: the end-to-end call of the paper's timing scope (Sec. 8.1.3: transfer of
+ * query vectors and ranges, then execution).  All pointers are HOST memory (pinned memory makes
+ * the copies asynchronous); copies in, searches, copies the results out and synchronises the
+ * stream.  Uses staging buffers owned by the index, grown on first use. */
+int frog_search_host(frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
+                     int nq, int k, int beam_width, int32_t* out_ids, float* out_dists, void* stream);
+
+/* Launch shape of the search kernel for the given beam width (for reporting): CTAs, threads per
+ * CTA, dynamic shared memory per CTA, query slots resident per SM. */
+int frog_search_launch_info(const frog_index_t* index, int beam_width, const frog_params_t* params,
+                            int* grid, int* block, int* smem_bytes, int* queries_per_sm);
+
+const char* frog_strerror(int code);
+
+/* cudaError_t value of the last failing CUDA call seen by this library on this thread. */
+int frog_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FROG_H_ */

@@ -1,0 +1,55 @@
+// Host-side definitions shared by the translation units of libfrog.so (not part of the ABI).
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "frog.h"
+
+struct frog_index {
+    frog_index_info_t info;
+    int32_t* d_sorted_attr = nullptr;
+    int32_t* d_rank2id = nullptr;
+    float* d_vectors = nullptr;      // n x d_pad, rank order
+    uint32_t* d_enc = nullptr;       // n x H x m
+    unsigned int* d_work = nullptr;  // scratch: work counter of the persistent kernel (+ spare words)
+    // staging for frog_search_host, grown on demand
+    void* d_stage = nullptr;
+    size_t stage_bytes = 0;
+    int sm_count = 0;
+};
+
+// Arguments of the search kernel (passed by value).
+struct FrogSearchArgs {
+    const int32_t* sorted_attr;
+    const int32_t* rank2id;
+    const float* vectors;
+    const uint32_t* enc;
+    int n, d, d_pad, H, m;
+    const float* queries;
+    const int32_t* lo;
+    const int32_t* hi;
+    int nq, k, ef_s, epn, B, max_iters, no_hotspot, hash_bits;
+    unsigned long long seed;
+    int32_t* out_ids;
+    float* out_dists;
+    uint32_t* status;
+    uint32_t* stats;
+    uint32_t* trace;
+    int trace_cap;
+    unsigned int* work_counter;
+};
+
+namespace froghost {
+void set_cuda_error(cudaError_t e);
+int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in, frog_params_t* out);
+}  // namespace froghost
+
+#define FROG_CUDA_TRY(expr)                                  \
+    do {                                                     \
+        cudaError_t _e = (expr);                             \
+        if (_e != cudaSuccess) {                             \
+            froghost::set_cuda_error(_e);                    \
+            return FROG_ERR_CUDA;                            \
+        }                                                    \
+    } while (0)

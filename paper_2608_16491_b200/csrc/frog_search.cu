@@ -1,0 +1,346 @@
+// frog_search / frog_search_ex: batched FROGSearch (paper Alg. 2) as one persistent kernel.
+//
+// Mapping.  Queries are independent (Sec. 7.1), so each WARP owns one query at a time and pulls
+// the next one from a global work counter; a CTA is just a bundle of such warps, they never
+// synchronise with each other.  Per-query state lives in that warp's slice of shared memory:
+// the candidate pool (sorted u64 keys), the new-candidate keys, the compacted EN array, the
+// query vector and the visited table.  Global memory holds the ENC array and the vectors; per
+// expansion the warp reads the hotspot rows of ENC(u) and the rows of the surviving ENs only.
+#include <cstdio>
+#include <cstring>
+
+#include "frog_device.cuh"
+#include "frog_internal.h"
+
+using namespace frogdev;
+
+namespace {
+
+constexpr int WARPS_PER_CTA = 4;
+
+struct WarpSmem {
+    uint64_t* pool;
+    uint64_t* nk;
+    uint32_t* en;
+    float4* q;
+    uint32_t* hash;
+};
+
+__host__ __device__ inline size_t warp_smem_bytes(int pool_slots, int d_pad, int hash_bits) {
+    return (size_t)pool_slots * 8 + 32 * 8 + 32 * 4 + (size_t)d_pad * 4 + ((size_t)4 << hash_bits);
+}
+
+// entry point j of a query range: stateless mixer of (seed, l_q, r_q, j), top 32 bits scaled
+// into [0, w) by a multiply-high (Alg. 2 line 3: uniform sample from [l_q, r_q])
+__device__ __forceinline__ uint32_t entry_point(unsigned long long seed, uint32_t l_q, uint32_t r_q, int j) {
+    unsigned long long x = seed ^ ((unsigned long long)l_q * 0x9E3779B97F4A7C15ull)
+                                ^ ((unsigned long long)r_q * 0xC2B2AE3D27D4EB4Full)
+                                ^ ((unsigned long long)(j + 1) * 0x165667B19E3779F9ull);
+    x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
+    x ^= x >> 27; x *= 0x94D049BB133111EBull;
+    x ^= x >> 31;
+    unsigned long long w = (unsigned long long)(r_q - l_q) + 1ull;
+    return l_q + (uint32_t)(((x >> 32) * w) >> 32);
+}
+
+// One batch of up to 32 candidate ranks (lane j < cnt holds cand): drop repeats inside the batch,
+// apply the visited check, compute the distances of the survivors, merge them into the pool.
+// Returns the first unexpanded pool position.
+template <int EPL>
+__device__ __forceinline__ int evaluate_batch(const FrogSearchArgs& A, const WarpSmem& S, uint32_t cand,
+                                              int cnt, bool use_hash, uint32_t new_flag, int lane,
+                                              uint32_t& n_dist, uint32_t& forgets) {
+    bool keep = lane < cnt;
+    if (use_hash) {
+        // the same vertex can sit in several layers of ENC(u): keep its first copy only
+        uint32_t same = __match_any_sync(FULL, keep ? cand : (0x80000000u | (uint32_t)lane));
+        keep = keep && ((__ffs(same) - 1) == lane);
+        if (keep) keep = visited_insert(S.hash, A.hash_bits, cand, forgets);
+    }
+    // compact the survivors to lanes 0..ns-1
+    uint32_t M = __ballot_sync(FULL, keep);
+    int ns = __popc(M);
+    __syncwarp();
+    if (keep) S.en[__popc(M & ((1u << lane) - 1u))] = cand;
+    __syncwarp();
+    uint32_t id = lane < ns ? S.en[lane] : 0u;
+    __syncwarp();
+    n_dist += ns;
+    int first = NO_POS;
+    for (int base = 0; base < max(ns, 1); base += 16) {
+        uint32_t sub_id = __shfl_sync(FULL, id, (base + lane) & 31);
+        int sub_ns = min(16, ns - base);
+        float d2 = sub_ns > 0 ? batch_dist2(A.vectors, A.d_pad, S.q, sub_id, sub_ns, lane) : 0.f;
+        uint64_t key = (lane < sub_ns) ? make_key(d2, sub_id, new_flag) : KEY_EMPTY;
+        first = merge_batch<EPL>(S.pool, S.nk, key, A.ef_s, lane);
+    }
+    return first;
+}
+
+template <int EPL, bool TRACE>
+__global__ void __launch_bounds__(WARPS_PER_CTA * 32)
+frog_search_kernel(const FrogSearchArgs A) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int lane = lane_id();
+    const int warp = threadIdx.x >> 5;
+    constexpr int POOL = 32 * EPL;
+    const size_t per_warp = warp_smem_bytes(POOL, A.d_pad, A.hash_bits);
+    unsigned char* base = smem_raw + per_warp * warp;
+    WarpSmem S;
+    S.pool = reinterpret_cast<uint64_t*>(base);
+    S.nk = S.pool + POOL;
+    S.en = reinterpret_cast<uint32_t*>(S.nk + 32);
+    S.q = reinterpret_cast<float4*>(S.en + 32);
+    S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<float*>(S.q) + A.d_pad);
+    const int hash_slots = 1 << A.hash_bits;
+
+    for (;;) {
+        int q = 0;
+        if (lane == 0) q = (int)atomicAdd(A.work_counter, 1u);
+        q = __shfl_sync(FULL, q, 0);
+        if (q >= A.nq) break;
+
+        // ---- per-query set-up ---------------------------------------------------------------
+        {
+            float* qf = reinterpret_cast<float*>(S.q);
+            const float* src = A.queries + (size_t)q * A.d;
+            for (int i = lane; i < A.d_pad; i += 32) qf[i] = i < A.d ? __ldg(src + i) : 0.f;
+            for (int i = lane; i < POOL; i += 32) S.pool[i] = KEY_EMPTY;
+        }
+        const int32_t lo = __ldg(A.lo + q), hi = __ldg(A.hi + q);
+        // Sec. 4: [lo, hi] -> rank interval [l_q, r_q]
+        const int l_q = warp_count_below(A.sorted_attr, A.n, lo, false, lane);
+        const int r_q = warp_count_below(A.sorted_attr, A.n, hi, true, lane) - 1;
+        const int w = (lo > hi) ? 0 : (r_q - l_q + 1);
+        uint32_t st = 0, n_exp = 0, n_rows = 0, n_en = 0, n_dist = 0, forgets = 0;
+        uint32_t trace_len = 0;
+        bool trace_ok = true;
+        uint32_t* trace_row = TRACE ? A.trace + (size_t)q * A.trace_cap : nullptr;
+        __syncwarp();
+
+        if (w <= 0) {
+            st |= FROG_ST_EMPTY;
+        } else if (w <= A.ef_s) {
+            // every valid object enters the pool: exact answer
+            st |= FROG_ST_EXACT;
+            for (int b0 = 0; b0 < w; b0 += 32) {
+                int cnt = min(32, w - b0);
+                evaluate_batch<EPL>(A, S, (uint32_t)(l_q + b0 + lane), cnt, false, 1u, lane, n_dist, forgets);
+            }
+        } else {
+            {
+                uint4* h4 = reinterpret_cast<uint4*>(S.hash);
+                const uint4 e4 = make_uint4(HASH_EMPTY, HASH_EMPTY, HASH_EMPTY, HASH_EMPTY);
+                for (int i = lane; i < (hash_slots >> 2); i += 32) h4[i] = e4;
+            }
+            int L_start, L_end;
+            hotspot_layers(l_q, r_q, A.H, A.n, L_start, L_end);          // Alg. 2 line 1
+            if (A.no_hotspot) { L_start = 0; L_end = A.H - 1; }
+            const int total = (L_end - L_start + 1) * A.m;
+            const uint32_t span = (uint32_t)(r_q - l_q);
+            __syncwarp();
+            // lines 2-5: entry points
+            uint32_t ep = lane < A.epn ? entry_point(A.seed, (uint32_t)l_q, (uint32_t)r_q, lane) : 0u;
+            int first = evaluate_batch<EPL>(A, S, ep, A.epn, true, 0u, lane, n_dist, forgets);
+            // lines 7-17
+            while (first < A.ef_s) {
+                if ((int)n_exp >= A.max_iters) { st |= FROG_ST_ITER_CAP; break; }
+                const uint32_t u = key_rank(S.pool[first]);               // line 8
+                __syncwarp();
+                if (lane == 0) S.pool[first] |= 1ull;                     // line 9
+                const uint32_t* hot = A.enc + ((size_t)u * A.H + L_start) * A.m;
+                int scanned;
+                int cnt = en_identify(hot, total, (uint32_t)l_q, span, A.B, S.en, lane, scanned);   // line 10
+                __syncwarp();
+                uint32_t cand = lane < cnt ? S.en[lane] : 0u;
+                ++n_exp;
+                n_rows += (scanned + A.m - 1) / A.m;
+                n_en += cnt;
+                if (TRACE) {
+                    // records are appended until the first one that does not fit
+                    if (trace_ok && trace_len + 2 + cnt <= (uint32_t)A.trace_cap - 1) {
+                        if (lane == 0) { trace_row[1 + trace_len] = u; trace_row[2 + trace_len] = (uint32_t)cnt; }
+                        if (lane < cnt) trace_row[3 + trace_len + lane] = cand;
+                        trace_len += 2 + cnt;
+                    } else {
+                        trace_ok = false;
+                    }
+                }
+                first = evaluate_batch<EPL>(A, S, cand, cnt, true, 0u, lane, n_dist, forgets);   // lines 11-17
+            }
+        }
+
+        // ---- line 18: first k of the pool ---------------------------------------------------
+        __syncwarp();
+        int got = 0;
+        for (int j = lane; j < A.k; j += 32) {
+            uint64_t key = S.pool[j];
+            int32_t oid = -1;
+            float dist = __int_as_float(0x7F800000);
+            if (key != KEY_EMPTY) {
+                oid = __ldg(A.rank2id + key_rank(key));
+                dist = __fsqrt_rn(key_dist2(key));
+                ++got;
+            }
+            A.out_ids[(size_t)q * A.k + j] = oid;
+            A.out_dists[(size_t)q * A.k + j] = dist;
+        }
+        got = __reduce_add_sync(FULL, got);
+        if (got < A.k) st |= FROG_ST_SHORT;
+        if (lane == 0) {
+            if (A.status) A.status[q] = st;
+            if (A.stats) {
+                uint32_t* srow = A.stats + 4 * (size_t)q;
+                srow[0] = n_exp; srow[1] = n_rows; srow[2] = n_en; srow[3] = n_dist;
+            }
+            if (TRACE) trace_row[0] = trace_len;
+        }
+        (void)forgets;
+        __syncwarp();
+    }
+}
+
+typedef void (*kernel_fn)(const FrogSearchArgs);
+
+template <bool TRACE>
+kernel_fn pick_kernel(int ef_s, int* pool_slots) {
+    if (ef_s <= 32) { *pool_slots = 32; return frog_search_kernel<1, TRACE>; }
+    if (ef_s <= 64) { *pool_slots = 64; return frog_search_kernel<2, TRACE>; }
+    if (ef_s <= 128) { *pool_slots = 128; return frog_search_kernel<4, TRACE>; }
+    if (ef_s <= 256) { *pool_slots = 256; return frog_search_kernel<8, TRACE>; }
+    *pool_slots = 512;
+    return frog_search_kernel<16, TRACE>;
+}
+
+struct LaunchPlan {
+    kernel_fn fn;
+    int grid, block, ctas_per_sm;
+    size_t smem;
+};
+
+int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, bool trace, int nq, LaunchPlan* out) {
+    int pool_slots = 0;
+    kernel_fn fn = trace ? pick_kernel<true>(beam_width, &pool_slots) : pick_kernel<false>(beam_width, &pool_slots);
+    size_t smem = warp_smem_bytes(pool_slots, ix->info.d_pad, P.hash_bits) * WARPS_PER_CTA;
+    if (smem > 227 * 1024) return FROG_ERR_UNSUPPORTED;
+    FROG_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    FROG_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)fn, WARPS_PER_CTA * 32, smem));
+    if (per_sm < 1) return FROG_ERR_UNSUPPORTED;
+    int grid = per_sm * ix->sm_count;
+    if (nq > 0) {
+        int need = (nq + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
+        if (grid > need) grid = need;
+    }
+    out->fn = fn;
+    out->grid = grid < 1 ? 1 : grid;
+    out->block = WARPS_PER_CTA * 32;
+    out->ctas_per_sm = per_sm;
+    out->smem = smem;
+    return FROG_OK;
+}
+
+}  // namespace
+
+namespace froghost {
+
+int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in, frog_params_t* out) {
+    frog_params_t P;
+    std::memset(&P, 0, sizeof(P));
+    if (in) P = *in;
+    if (P.epn == 0) P.epn = 16;
+    if (P.budget == 0) P.budget = 16;
+    if (P.max_iters == 0) P.max_iters = 16 * beam_width;
+    if (P.epn < 1 || P.epn > FROG_MAX_BUDGET || P.budget < 1 || P.budget > FROG_MAX_BUDGET || P.max_iters < 1)
+        return FROG_ERR_INVALID_ARG;
+    if (P.hash_bits == 0) {
+        // about 16 evaluated vertices per beam slot, at most half full
+        int want = 16 * beam_width;
+        int bits = 9;
+        while ((1 << bits) < want && bits < 13) ++bits;
+        P.hash_bits = bits;
+    }
+    if (P.hash_bits < 6 || P.hash_bits > 15) return FROG_ERR_INVALID_ARG;
+    (void)ix;
+    *out = P;
+    return FROG_OK;
+}
+
+}  // namespace froghost
+
+extern "C" int frog_search_launch_info(const frog_index_t* index, int beam_width, const frog_params_t* params,
+                                       int* grid, int* block, int* smem_bytes, int* queries_per_sm) {
+    if (!index || beam_width < 1 || beam_width > FROG_MAX_BEAM_WIDTH) return FROG_ERR_INVALID_ARG;
+    frog_params_t P;
+    int rc = froghost::resolve_params(index, beam_width, params, &P);
+    if (rc) return rc;
+    FROG_CUDA_TRY(cudaSetDevice(index->info.device));
+    LaunchPlan plan;
+    rc = plan_launch(index, beam_width, P, false, 0, &plan);
+    if (rc) return rc;
+    if (grid) *grid = plan.grid;
+    if (block) *block = plan.block;
+    if (smem_bytes) *smem_bytes = (int)plan.smem;
+    if (queries_per_sm) *queries_per_sm = plan.ctas_per_sm * WARPS_PER_CTA;
+    return FROG_OK;
+}
+
+extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
+                              int nq, int k, int beam_width, const frog_params_t* params,
+                              int32_t* out_ids, float* out_dists, uint32_t* status, uint32_t* stats,
+                              uint32_t* trace, int trace_cap, void* stream) {
+    if (!index || nq < 0) return FROG_ERR_INVALID_ARG;
+    if (k < 1 || beam_width < 1 || beam_width > FROG_MAX_BEAM_WIDTH || k > beam_width) return FROG_ERR_INVALID_ARG;
+    if (trace && trace_cap < 4) return FROG_ERR_INVALID_ARG;
+    if (nq == 0) return FROG_OK;
+    if (!queries || !lo || !hi || !out_ids || !out_dists) return FROG_ERR_INVALID_ARG;
+    frog_params_t P;
+    int rc = froghost::resolve_params(index, beam_width, params, &P);
+    if (rc) return rc;
+    FROG_CUDA_TRY(cudaSetDevice(index->info.device));
+    LaunchPlan plan;
+    rc = plan_launch(index, beam_width, P, trace != nullptr, nq, &plan);
+    if (rc) return rc;
+
+    FrogSearchArgs A;
+    A.sorted_attr = index->d_sorted_attr;
+    A.rank2id = index->d_rank2id;
+    A.vectors = index->d_vectors;
+    A.enc = index->d_enc;
+    A.n = (int)index->info.n;
+    A.d = index->info.d;
+    A.d_pad = index->info.d_pad;
+    A.H = index->info.H;
+    A.m = index->info.m;
+    A.queries = queries;
+    A.lo = lo;
+    A.hi = hi;
+    A.nq = nq;
+    A.k = k;
+    A.ef_s = beam_width;
+    A.epn = P.epn;
+    A.B = P.budget;
+    A.max_iters = P.max_iters;
+    A.no_hotspot = P.no_hotspot;
+    A.hash_bits = P.hash_bits;
+    A.seed = P.seed;
+    A.out_ids = out_ids;
+    A.out_dists = out_dists;
+    A.status = status;
+    A.stats = stats;
+    A.trace = trace;
+    A.trace_cap = trace_cap;
+    A.work_counter = index->d_work;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    FROG_CUDA_TRY(cudaMemsetAsync(index->d_work, 0, sizeof(unsigned int), s));
+    plan.fn<<<plan.grid, plan.block, plan.smem, s>>>(A);
+    FROG_CUDA_TRY(cudaGetLastError());
+    return FROG_OK;
+}
+
+extern "C" int frog_search(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
+                           int nq, int k, int beam_width, int32_t* out_ids, float* out_dists, void* stream) {
+    return frog_search_ex(index, queries, lo, hi, nq, k, beam_width, nullptr, out_ids, out_dists,
+                          nullptr, nullptr, nullptr, 0, stream);
+}

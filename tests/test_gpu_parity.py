@@ -1,0 +1,233 @@
+"""CUDA search path against the CPU oracle, element by element, through the C ABI."""
+import ctypes
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+def _dev(x):
+    return torch.from_numpy(np.ascontiguousarray(x)).cuda()
+
+
+def _gpu_search(frog, gix, wl_q, lo, hi, k, ef, trace_cap=0, **params):
+    nq = wl_q.shape[0]
+    q, tlo, thi = _dev(wl_q), _dev(lo), _dev(hi)
+    status = torch.zeros(nq, dtype=torch.int32, device="cuda")
+    stats = torch.zeros((nq, 4), dtype=torch.int32, device="cuda")
+    trace = torch.zeros((nq, trace_cap), dtype=torch.int32, device="cuda") if trace_cap else None
+    p = frog.Params(**params) if params else None
+    ids, dists = gix.search(q, tlo, thi, k, ef, params=p, status=status, stats=stats, trace=trace)
+    torch.cuda.synchronize()
+    return (ids.cpu().numpy(), dists.cpu().numpy(), status.cpu().numpy().view(np.uint32),
+            stats.cpu().numpy().view(np.uint32), None if trace is None else trace.cpu().numpy().view(np.uint32))
+
+
+def _assert_parity(got, ref, check_dist_count=True):
+    ids, dists, status, stats, trace = got
+    # returned ids: bit-exact; distances: identical arithmetic order, so also bit-exact, and in any
+    # case within the 1e-4 relative tolerance the parity target states
+    assert np.array_equal(ids, ref.ids)
+    fin = np.isfinite(ref.dists)
+    assert np.array_equal(np.isfinite(dists), fin)
+    assert np.allclose(dists[fin], ref.dists[fin], rtol=1e-4, atol=0)
+    assert np.array_equal(dists[fin], ref.dists[fin])
+    assert np.array_equal(status, ref.status)
+    # expansions, ENC rows read, ENs admitted: bit-exact (integer work)
+    assert np.array_equal(stats[:, :3], ref.stats[:, :3])
+    # distance evaluations: equal unless the GPU's bounded visited table forgot an entry, which
+    # can only add evaluations
+    assert np.all(stats[:, 3] >= ref.stats[:, 3])
+    if check_dist_count:
+        assert np.array_equal(stats[:, 3], ref.stats[:, 3])
+    if trace is not None and ref.trace is not None:
+        assert np.array_equal(trace, ref.trace)         # every EN list of every expansion
+
+
+@pytest.fixture(scope="module")
+def tiny_gpu(libs, tiny):
+    wl, path, ix = tiny
+    gix = libs.Index.load(path, 0)
+    yield wl, ix, gix
+    gix.close()
+
+
+@pytest.mark.parametrize("ef", [16, 24, 32, 48, 64, 96, 128, 192, 256, 512])
+def test_tiny_matches_oracle_at_every_beam_width(libs, tiny_gpu, ef):
+    wl, ix, gix = tiny_gpu
+    ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, ef, trace_cap=40000 if ef <= 128 else 0)
+    got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, wl.k, ef, trace_cap=40000 if ef <= 128 else 0)
+    _assert_parity(got, ref)
+
+
+def test_tiny_plain_call_equals_ex_call(libs, tiny_gpu):
+    wl, ix, gix = tiny_gpu
+    q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
+    ids, dists = gix.search(q, lo, hi, wl.k, 64)
+    torch.cuda.synchronize()
+    ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 64)
+    assert np.array_equal(ids.cpu().numpy(), ref.ids)
+    assert np.array_equal(dists.cpu().numpy(), ref.dists)
+
+
+@pytest.mark.parametrize("params", [dict(epn=1), dict(epn=32), dict(budget=4), dict(budget=32),
+                                    dict(no_hotspot=1), dict(seed=12345), dict(max_iters=7),
+                                    dict(epn=7, budget=9, seed=3)])
+def test_tiny_parameter_variants(libs, tiny_gpu, params):
+    wl, ix, gix = tiny_gpu
+    okw = dict(epn=params.get("epn", 16), B=params.get("budget", 16), seed=params.get("seed", 0),
+               no_hotspot=bool(params.get("no_hotspot", 0)), max_iters=params.get("max_iters", 0))
+    ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 48, trace_cap=20000, **okw)
+    got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, wl.k, 48, trace_cap=20000, **params)
+    _assert_parity(got, ref)
+
+
+def test_k_equals_beam_and_k_one(libs, tiny_gpu):
+    wl, ix, gix = tiny_gpu
+    for k, ef in ((32, 32), (1, 16), (100, 128), (64, 64)):
+        ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef)
+        got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, k, ef)
+        _assert_parity(got, ref)
+
+
+def test_edge_ranges(libs, tiny_gpu):
+    """Empty, inverted, single-object, fewer-than-k, exactly-beam-sized and full ranges."""
+    wl, ix, gix = tiny_gpu
+    srt = np.asarray(ix.sorted_attr)
+    lo = np.array([5, -100, srt[0], srt[10], srt[100], srt[100], -2**31, srt[9999], srt[0]], np.int32)
+    hi = np.array([4, -50, srt[0], srt[14], srt[131], srt[132], 2**31 - 1, 2**31 - 1, srt[9999]], np.int32)
+    Q = wl.queries[: lo.size]
+    ref = oracle.search(ix, Q, lo, hi, 10, 32, trace_cap=8000)
+    got = _gpu_search(libs, gix, Q, lo, hi, 10, 32, trace_cap=8000)
+    _assert_parity(got, ref)
+    assert ref.status[0] & oracle.ST_EMPTY and ref.status[1] & oracle.ST_EMPTY
+    assert ref.status[4] & oracle.ST_EXACT and not (ref.status[5] & oracle.ST_EXACT)
+
+
+def test_small_visited_table_changes_work_not_results(libs, tiny_gpu):
+    """A visited table far too small forgets entries: more distance evaluations, same answers."""
+    wl, ix, gix = tiny_gpu
+    ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 64, trace_cap=20000)
+    got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, wl.k, 64, trace_cap=20000, hash_bits=6)
+    _assert_parity(got, ref, check_dist_count=False)
+    assert got[3][:, 3].sum() > ref.stats[:, 3].sum()
+
+
+def test_empty_batch_and_argument_errors(libs, tiny_gpu):
+    wl, ix, gix = tiny_gpu
+    q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
+    ids, _ = gix.search(q[:0], lo[:0], hi[:0], 10, 32)
+    assert ids.shape == (0, 10)
+    for k, ef in ((0, 32), (33, 32), (10, 0), (10, 513)):
+        with pytest.raises(libs.FrogError) as e:
+            gix.search(q, lo, hi, k, ef)
+        assert e.value.code == 1
+    with pytest.raises(libs.FrogError):
+        gix.search(q, lo, hi, 10, 32, params=libs.Params(epn=33))
+    # a failed call leaves the index usable
+    ids, _ = gix.search(q, lo, hi, 10, 32)
+    torch.cuda.synchronize()
+    assert ids.shape == (wl.nq, 10)
+
+
+def test_exact_search_matches_definition(libs, tiny_gpu):
+    wl, ix, gix = tiny_gpu
+    q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
+    for k in (1, 10, 100):
+        ids, dists = gix.exact_search(q, lo, hi, k)
+        torch.cuda.synchronize()
+        ref_ids, ref_d, _ = oracle.exact_slab(ix, wl.queries, wl.lo, wl.hi, k, mode=1)
+        assert np.array_equal(ids.cpu().numpy(), ref_ids)
+        assert np.array_equal(dists.cpu().numpy(), ref_d)
+        # against the float64 definition: same ids except at near-ties, distances within 1e-4
+        def_ids, def_d = oracle.exact_scan(wl.vectors, wl.attrs, wl.queries, wl.lo, wl.hi, k, mode=0)
+        fin = np.isfinite(def_d)
+        assert np.allclose(dists.cpu().numpy()[fin], def_d[fin], rtol=1e-4)
+        assert (ids.cpu().numpy() == def_ids).mean() > 0.999
+
+
+def test_host_buffer_call_matches(libs, tiny_gpu):
+    wl, ix, gix = tiny_gpu
+    ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 64)
+    ids, dists = gix.search_host(torch.from_numpy(wl.queries).pin_memory(),
+                                 torch.from_numpy(wl.lo).pin_memory(),
+                                 torch.from_numpy(wl.hi).pin_memory(), wl.k, 64)
+    assert np.array_equal(ids.numpy(), ref.ids) and np.array_equal(dists.numpy(), ref.dists)
+    # a second, larger call regrows the staging area
+    reps = 3
+    Q = np.tile(wl.queries, (reps, 1))
+    ids, dists = gix.search_host(Q, np.tile(wl.lo, reps), np.tile(wl.hi, reps), wl.k, 64)
+    assert np.array_equal(ids.numpy(), np.tile(ref.ids, (reps, 1)))
+
+
+def test_recall_within_tolerance_of_oracle(libs, tiny_gpu):
+    wl, ix, gix = tiny_gpu
+    gt, _, _ = oracle.exact_slab(ix, wl.queries, wl.lo, wl.hi, wl.k, mode=0)
+    for ef in (16, 64):
+        ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, ef)
+        got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, wl.k, ef)
+        assert abs(oracle.recall(got[0], gt) - oracle.recall(ref.ids, gt)) <= 0.005
+
+
+# ---- the other workload shapes at sizes the oracle finishes in seconds ------------------------
+@pytest.mark.parametrize("name,n,nq", [("sift", 60_000, 300), ("deep1m", 50_000, 300),
+                                        ("deep10m", 70_001, 300), ("text", 20_000, 150)])
+def test_scaled_workloads_match_oracle(libs, cache_dir, name, n, nq):
+    from conftest import build_scaled
+    wl, path, ix = build_scaled(libs, cache_dir, name, n, nq)
+    gix = libs.Index.load(path, 0)
+    try:
+        for ef, k in ((32, 10), (100, 100)):
+            ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef, trace_cap=30000)
+            got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, k, ef, trace_cap=30000)
+            _assert_parity(got, ref)
+        q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
+        ids, dists = gix.exact_search(q, lo, hi, 10)
+        torch.cuda.synchronize()
+        ref_ids, ref_d, _ = oracle.exact_slab(ix, wl.queries, wl.lo, wl.hi, 10, mode=1)
+        assert np.array_equal(ids.cpu().numpy(), ref_ids) and np.array_equal(dists.cpu().numpy(), ref_d)
+    finally:
+        gix.close()
+
+
+def test_odd_dimension(libs, cache_dir):
+    rng = np.random.default_rng(2)
+    V = rng.standard_normal((3000, 10)).astype(np.float32)
+    a = rng.integers(0, 500, 3000).astype(np.int32)
+    path = os.path.join(cache_dir, "odd_gpu.idx")
+    libs.build_index(V, a, path, n_inv=5)
+    ix = oracle.load_index(path)
+    gix = libs.Index.load(path, 0)
+    Q = rng.standard_normal((64, 10)).astype(np.float32)
+    lo = rng.integers(0, 400, 64).astype(np.int32)
+    hi = (lo + rng.integers(0, 100, 64)).astype(np.int32)
+    ref = oracle.search(ix, Q, lo, hi, 5, 32)
+    got = _gpu_search(libs, gix, Q, lo, hi, 5, 32)
+    _assert_parity(got, ref)
+    gix.close()
+
+
+def test_index_info_and_from_host(libs, tiny):
+    wl, path, ix = tiny
+    gix = libs.Index.load(path, 0)
+    info = gix.info
+    assert (info.n, info.d, info.d_pad, info.H, info.m) == (ix.n, ix.d, ix.d_pad, ix.H, ix.m)
+    assert info.device_bytes >= ix.n * (8 + 4 * ix.d_pad + 4 * ix.H * ix.m)
+    h = ctypes.c_void_p()
+    shape = libs.IndexInfo(n=ix.n, d=ix.d, d_pad=ix.d_pad, H=ix.H, m=ix.m)
+    arrs = [np.ascontiguousarray(a) for a in (ix.sorted_attr, ix.rank2id, ix.vectors, ix.enc)]
+    rc = libs._lib.frog_index_from_host(*[a.ctypes.data_as(ctypes.c_void_p) for a in arrs],
+                                        ctypes.byref(shape), 0, ctypes.byref(h))
+    assert rc == 0
+    g2 = libs.Index(h)
+    ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 32)
+    got = _gpu_search(libs, g2, wl.queries, wl.lo, wl.hi, wl.k, 32)
+    _assert_parity(got, ref)
+    g2.close()
+    gix.close()
