@@ -73,6 +73,8 @@ typedef struct {
 #define FROG_ST_EXACT 2u     /* range holds <= beam_width objects: answered by exact scan */
 #define FROG_ST_ITER_CAP 4u  /* expansion cap hit; the current pool was returned */
 #define FROG_ST_SHORT 8u     /* fewer than k results; tail is padding */
+#define FROG_ST_FORGOT 16u   /* the visited table overflowed and dropped entries: some distances were
+                                evaluated twice; the results are unaffected */
 
 /* frog_index_load: read an index file, copy its four arrays to `device`, return a handle.
  * (Paper Sec. 8.1.3: index and database stay resident in GPU memory.)  Host pointer in, the

@@ -24,7 +24,7 @@ _LIB_SEARCH = os.path.join(_HERE, "libfrog.so")
 _LIB_BUILD = os.path.join(_HERE, "libfrog_build.so")
 
 FROG_MAX_BEAM_WIDTH = 512
-ST_EMPTY, ST_EXACT, ST_ITER_CAP, ST_SHORT = 1, 2, 4, 8
+ST_EMPTY, ST_EXACT, ST_ITER_CAP, ST_SHORT, ST_FORGOT = 1, 2, 4, 8, 16
 
 
 class FrogError(RuntimeError):

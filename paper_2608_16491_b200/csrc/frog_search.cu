@@ -187,6 +187,7 @@ frog_search_kernel(const FrogSearchArgs A) {
         }
         got = __reduce_add_sync(FULL, got);
         if (got < A.k) st |= FROG_ST_SHORT;
+        if (__any_sync(FULL, forgets != 0)) st |= FROG_ST_FORGOT;   // counted per lane
         if (lane == 0) {
             if (A.status) A.status[q] = st;
             if (A.stats) {
@@ -195,7 +196,6 @@ frog_search_kernel(const FrogSearchArgs A) {
             }
             if (TRACE) trace_row[0] = trace_len;
         }
-        (void)forgets;
         __syncwarp();
     }
 }

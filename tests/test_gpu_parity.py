@@ -29,7 +29,14 @@ def _gpu_search(frog, gix, wl_q, lo, hi, k, ef, trace_cap=0, **params):
             stats.cpu().numpy().view(np.uint32), None if trace is None else trace.cpu().numpy().view(np.uint32))
 
 
-def _assert_parity(got, ref, check_dist_count=True):
+def _default_slots(ef):
+    bits = 9
+    while (1 << bits) < 16 * ef and bits < 13:
+        bits += 1
+    return 1 << bits
+
+
+def _assert_parity(got, ref, check_dist_count=True, slots=None):
     ids, dists, status, stats, trace = got
     # returned ids: bit-exact; distances: identical arithmetic order, so also bit-exact, and in any
     # case within the 1e-4 relative tolerance the parity target states
@@ -38,14 +45,19 @@ def _assert_parity(got, ref, check_dist_count=True):
     assert np.array_equal(np.isfinite(dists), fin)
     assert np.allclose(dists[fin], ref.dists[fin], rtol=1e-4, atol=0)
     assert np.array_equal(dists[fin], ref.dists[fin])
-    assert np.array_equal(status, ref.status)
+    forgot = (status & 16) != 0       # GPU-only bit: visited table overflowed (work, not results)
+    assert np.array_equal(status & ~np.uint32(16), ref.status)
     # expansions, ENC rows read, ENs admitted: bit-exact (integer work)
     assert np.array_equal(stats[:, :3], ref.stats[:, :3])
     # distance evaluations: equal unless the GPU's bounded visited table forgot an entry, which
     # can only add evaluations
     assert np.all(stats[:, 3] >= ref.stats[:, 3])
-    if check_dist_count:
-        assert np.array_equal(stats[:, 3], ref.stats[:, 3])
+    assert np.array_equal(stats[~forgot, 3], ref.stats[~forgot, 3])
+    if slots is not None:
+        # below half load a 24-slot probe run is out of reach: nothing may be forgotten
+        assert not forgot[ref.stats[:, 3] <= slots // 2].any()
+    elif check_dist_count:
+        assert forgot.mean() <= 0.02
     if trace is not None and ref.trace is not None:
         assert np.array_equal(trace, ref.trace)         # every EN list of every expansion
 
@@ -105,7 +117,7 @@ def test_edge_ranges(libs, tiny_gpu):
     Q = wl.queries[: lo.size]
     ref = oracle.search(ix, Q, lo, hi, 10, 32, trace_cap=8000)
     got = _gpu_search(libs, gix, Q, lo, hi, 10, 32, trace_cap=8000)
-    _assert_parity(got, ref)
+    _assert_parity(got, ref, check_dist_count=False)
     assert ref.status[0] & oracle.ST_EMPTY and ref.status[1] & oracle.ST_EMPTY
     assert ref.status[4] & oracle.ST_EXACT and not (ref.status[5] & oracle.ST_EXACT)
 
@@ -117,6 +129,7 @@ def test_small_visited_table_changes_work_not_results(libs, tiny_gpu):
     got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, wl.k, 64, trace_cap=20000, hash_bits=6)
     _assert_parity(got, ref, check_dist_count=False)
     assert got[3][:, 3].sum() > ref.stats[:, 3].sum()
+    assert (got[2] & 16).any()
 
 
 def test_empty_batch_and_argument_errors(libs, tiny_gpu):
@@ -186,7 +199,7 @@ def test_scaled_workloads_match_oracle(libs, cache_dir, name, n, nq):
         for ef, k in ((32, 10), (100, 100)):
             ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef, trace_cap=30000)
             got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, k, ef, trace_cap=30000)
-            _assert_parity(got, ref)
+            _assert_parity(got, ref, slots=_default_slots(ef))
         q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
         ids, dists = gix.exact_search(q, lo, hi, 10)
         torch.cuda.synchronize()
