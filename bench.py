@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark of the FROG search hot path: mixed-selectivity QPS at recall@10 >= 0.95 on one B200,
+with the achieved fraction of the HBM roofline and the CPU oracle timed beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one frog_search call over the whole query batch (every row of the hot path: endpoint
+lookup, hotspot localization, entry points, the expansion loop with EN identification, lazy hash
+check, vector gather + L2, sort/merge, output).  The index and the queries are resident in HBM
+when the timed region starts; the ``e2e`` figure repeats the measurement through the host-buffer
+call, transfers included.  With N > 1 every rank holds a full replica and answers its own copy of
+the batch (no data-path collective).  ``--impl reference`` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "mixed-selectivity QPS at recall@10>=0.95"
+UNIT = "queries/s"
+SWEEP = [16, 24, 32, 48, 64, 96, 128, 192, 256, 384, 512]
+RECALL_TARGET = 0.95
+HBM_FALLBACK_GBS = 6650.0
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return HBM_FALLBACK_GBS, "fallback"
+
+
+def prepare_index(frog, wl, cache_dir):
+    """Build (or reuse) the index file of a workload.  The cache is an optimisation only."""
+    os.makedirs(cache_dir, exist_ok=True)
+    from paper_2608_16491_b200 import build as b
+    h = hashlib.sha1()
+    h.update(open(os.path.join(b.CSRC, "frog_build.cpp"), "rb").read())
+    h.update(open(os.path.join(ROOT, "datagen", "__init__.py"), "rb").read())
+    tag = h.hexdigest()[:12]
+    path = os.path.join(cache_dir, f"{wl.name}_{wl.n}_{tag}.idx")
+    secs = 0.0
+    if not os.path.exists(path):
+        t = time.time()
+        tmp = path + f".tmp{os.getpid()}"
+        frog.build_index(wl.vectors, wl.attrs, tmp, seed=wl.seed)
+        os.replace(tmp, path)
+        secs = time.time() - t
+    return path, secs
+
+
+def recall_at_k(ids: np.ndarray, gt: np.ndarray) -> float:
+    valid = gt >= 0
+    hit = (ids[:, :, None] == gt[:, None, :]) & valid[:, None, :]
+    per_q = hit.any(axis=1).sum(axis=1)
+    denom = valid.sum(axis=1)
+    ok = denom > 0
+    return float((per_q[ok] / denom[ok]).mean())
+
+
+def recall_tie_aware(dists: np.ndarray, gt_d: np.ndarray) -> float:
+    fin = np.isfinite(gt_d)
+    denom = fin.sum(axis=1)
+    kth = np.where(fin, gt_d, -np.inf).max(axis=1)
+    hit = (dists <= kth[:, None] * (1 + 1e-6)) & np.isfinite(dists)
+    ok = denom > 0
+    return float((np.minimum(hit.sum(axis=1), denom)[ok] / denom[ok]).mean())
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device: int):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50", "-i", str(device)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+
+    def summary(self, t0, t1):
+        rows = [s for t, s in self.samples if t0 <= t <= t1] or [s for _, s in self.samples]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except Exception:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v == "Active":
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def algorithmic_bytes(stats: np.ndarray, n: int, d: int, d_pad: int, m: int, k: int) -> float:
+    """Bytes the method must move per batch: query vector, endpoint probes, ENC rows scanned,
+    vectors whose distance is evaluated, and the result rows."""
+    nq = stats.shape[0]
+    per_q = 4 * d + 8 * math.ceil(math.log2(max(n, 2))) + 8 * k
+    return float(nq * per_q + 4.0 * m * stats[:, 1].astype(np.float64).sum()
+                 + 4.0 * d_pad * stats[:, 3].astype(np.float64).sum())
+
+
+def ensure_built():
+    """Compile the libraries if they are missing (rank 0 builds, the others wait for the files)."""
+    from paper_2608_16491_b200 import build as b
+    rank = int(os.environ.get("RANK", "0"))
+    missing = [p for p in (b.LIB_SEARCH, b.LIB_BUILD) if not os.path.exists(p)]
+    if missing and rank == 0:
+        b.build_all()
+    t0 = time.time()
+    while any(not os.path.exists(p) for p in (b.LIB_SEARCH, b.LIB_BUILD)):
+        if time.time() - t0 > 900:
+            raise SystemExit("shared libraries missing and not built within 15 minutes")
+        time.sleep(1.0)
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on the host cores: K steps over a bounded query sample."""
+    from paper_2608_16491_b200 import replicas
+    rank, _, ws = replicas.world()
+    if rank != 0:
+        return
+    import datagen
+    import oracle
+    import paper_2608_16491_b200 as frog
+    wl = datagen.make_workload(args.workload, n=args.n or None, nq=args.nq or None)
+    path, build_s = prepare_index(frog, wl, args.cache_dir)
+    ix = oracle.load_index(path)
+    S = min(args.ref_sample, wl.nq)
+    Q, lo, hi = wl.queries[:S], wl.lo[:S], wl.hi[:S]
+    beam = args.beam
+    if beam <= 0:
+        probe = min(300, S)
+        gt, _, _ = oracle.exact_slab(ix, Q[:probe], lo[:probe], hi[:probe], wl.k, mode=0)
+        beam = SWEEP[-1]
+        for ef in SWEEP:
+            r = oracle.search(ix, Q[:probe], lo[:probe], hi[:probe], wl.k, ef)
+            if recall_at_k(r.ids, gt) >= RECALL_TARGET:
+                beam = ef
+                break
+    for _ in range(args.warmup):
+        oracle.search(ix, Q, lo, hi, wl.k, beam)
+    t0 = time.perf_counter()
+    threads = 1
+    for _ in range(args.steps):
+        threads = oracle.search(ix, Q, lo, hi, wl.k, beam).threads
+    dt = time.perf_counter() - t0
+    qps = S * args.steps / dt
+    out = {
+        "impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": f"{wl.name}: n={wl.n} d={wl.d} nq={wl.nq} k={wl.k} mixed selectivity",
+                   "beam_width": beam, "sample_queries": S},
+        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": f"first {S} of {wl.nq} queries per step, beam_width={beam}"},
+        "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def run_ours(args):
+    import torch
+    from paper_2608_16491_b200 import replicas
+    rank, local_rank, ws = replicas.world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the search path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    replicas.init("nccl")
+    import datagen
+    import paper_2608_16491_b200 as frog
+
+    t = time.time()
+    wl = datagen.make_workload(args.workload, n=args.n or None, nq=args.nq or None)
+    gen_s = time.time() - t
+    if rank == 0:
+        path, build_s = prepare_index(frog, wl, args.cache_dir)
+    replicas.barrier()
+    if rank != 0:
+        path, build_s = prepare_index(frog, wl, args.cache_dir)
+    t = time.time()
+    ix = frog.Index.load(path, local_rank)
+    load_s = time.time() - t
+    info = ix.info
+    log(f"[bench] workload {wl.name} n={wl.n} d={wl.d} nq={wl.nq}: gen {gen_s:.1f}s build {build_s:.1f}s load {load_s:.1f}s")
+
+    q = torch.from_numpy(wl.queries).to(dev)
+    lo = torch.from_numpy(wl.lo).to(dev)
+    hi = torch.from_numpy(wl.hi).to(dev)
+    nq, k = wl.nq, wl.k
+    out_ids = torch.empty((nq, k), dtype=torch.int32, device=dev)
+    out_d = torch.empty((nq, k), dtype=torch.float32, device=dev)
+    stats = torch.zeros((nq, 4), dtype=torch.int32, device=dev)
+    status = torch.zeros(nq, dtype=torch.int32, device=dev)
+
+    # ground truth (exact filtered kNN by slab scan on the GPU; parity-tested against the oracle)
+    gt_ids, gt_d = ix.exact_search(q, lo, hi, k)
+    torch.cuda.synchronize()
+    gt_ids_h, gt_d_h = gt_ids.cpu().numpy(), gt_d.cpu().numpy()
+
+    # beam-width sweep: smallest ef_s reaching the recall target
+    sweep = []
+    beam = args.beam
+    for ef in ([beam] if beam > 0 else SWEEP):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ix.search(q, lo, hi, k, ef, out_ids=out_ids, out_dists=out_d)   # warm
+        e0.record()
+        ix.search(q, lo, hi, k, ef, out_ids=out_ids, out_dists=out_d)
+        e1.record()
+        torch.cuda.synchronize()
+        rec = recall_at_k(out_ids.cpu().numpy(), gt_ids_h)
+        rec_t = recall_tie_aware(out_d.cpu().numpy(), gt_d_h)
+        sweep.append({"beam_width": ef, "recall": round(rec, 4), "recall_tie_aware": round(rec_t, 4),
+                      "qps": round(nq / (e0.elapsed_time(e1) * 1e-3))})
+        log(f"[bench] ef_s={ef}: recall@{k}={rec:.4f} (tie-aware {rec_t:.4f}) {sweep[-1]['qps']} q/s")
+        if beam <= 0 and rec >= RECALL_TARGET:
+            beam = ef
+            break
+    if beam <= 0:
+        beam = SWEEP[-1]
+    chosen = [s for s in sweep if s["beam_width"] == beam][0]
+
+    # counters of the chosen configuration -> algorithmic bytes per launch
+    ix.search(q, lo, hi, k, beam, out_ids=out_ids, out_dists=out_d, status=status, stats=stats)
+    torch.cuda.synchronize()
+    st = stats.cpu().numpy().view(np.uint32)
+    alg_bytes = algorithmic_bytes(st, info.n, info.d, info.d_pad, info.m, k)
+    launch = ix.launch_info(beam)
+
+    # ---- timed region: K launches, device-resident inputs ----------------------------------------
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    stream = torch.cuda.current_stream()
+    for _ in range(max(args.warmup, 3)):
+        ix.search(q, lo, hi, k, beam, out_ids=out_ids, out_dists=out_d)
+    torch.cuda.synchronize()
+    replicas.barrier()
+    torch.cuda.synchronize()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    t_wall0 = time.time()
+    evs[0].record(stream)
+    for i in range(args.steps):
+        ix.search(q, lo, hi, k, beam, out_ids=out_ids, out_dists=out_d)
+        evs[i + 1].record(stream)
+    torch.cuda.synchronize()
+    replicas.barrier()
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    total_ms = evs[0].elapsed_time(evs[-1])
+    per_launch_ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
+    total_ms_max = replicas.max_over_ranks(total_ms, dev)
+    clocks = sampler.summary(t_wall0, t_wall1) if sampler else None
+
+    # ---- end to end: host buffers in, host buffers out, transfers inside the timed region ----------
+    hq = torch.from_numpy(wl.queries).pin_memory()
+    hlo = torch.from_numpy(wl.lo).pin_memory()
+    hhi = torch.from_numpy(wl.hi).pin_memory()
+    h_ids = torch.empty((nq, k), dtype=torch.int32).pin_memory()
+    h_d = torch.empty((nq, k), dtype=torch.float32).pin_memory()
+    for _ in range(3):
+        ix.search_host(hq, hlo, hhi, k, beam, out_ids=h_ids, out_dists=h_d)
+    replicas.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        ix.search_host(hq, hlo, hhi, k, beam, out_ids=h_ids, out_dists=h_d)
+    e2e_s = time.perf_counter() - t0
+    replicas.barrier()
+    e2e_s_max = replicas.max_over_ranks(e2e_s, dev)
+    if sampler:
+        sampler.stop()
+    e2e_same = bool(np.array_equal(h_ids.numpy(), out_ids.cpu().numpy()))
+
+    if rank != 0:
+        return
+    peak, peak_src = measured_hbm_peak()
+    mean_launch_ms = float(np.mean(per_launch_ms))
+    achieved = alg_bytes / (mean_launch_ms * 1e-3) / 1e9
+    value = ws * nq * args.steps / (total_ms_max * 1e-3)
+
+    # ---- CPU oracle on the host cores, bounded sample; doubles as a parity check ------------------
+    cpu = None
+    if not args.no_cpu_baseline:
+        import oracle
+        oix = oracle.load_index(path)
+        S = min(args.cpu_sample, nq)
+        t0 = time.perf_counter()
+        ref = oracle.search(oix, wl.queries[:S], wl.lo[:S], wl.hi[:S], k, beam)
+        dt = time.perf_counter() - t0
+        ids_h = out_ids.cpu().numpy()[:S]
+        cpu = {"value": S / dt, "unit": UNIT, "cores": ref.threads, "kind": "oracle",
+               "sample": f"first {S} of {nq} queries, beam_width={beam}, one pass",
+               "ids_equal_to_gpu": bool(np.array_equal(ids_h, ref.ids)),
+               "counters_equal_to_gpu": bool(np.array_equal(st[:S, :3], ref.stats[:, :3]))}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ws, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{wl.name}: n={wl.n} d={wl.d} nq={wl.nq} k={k} mixed selectivity "
+                               f"(width fraction log-uniform 2^-10..1)",
+                   "beam_width": beam, "recall_at_10": chosen["recall"],
+                   "recall_tie_aware": chosen["recall_tie_aware"], "epn": 16, "budget": 16,
+                   "index": {"H": info.H, "m": info.m, "bytes": info.device_bytes, "build_seconds": round(build_s, 1)},
+                   "l2": "inputs larger than L2 (1.4 GB index, ~%.1f GB gathered per launch)" % (alg_bytes / 1e9),
+                   "parallelism": "replicas" if ws > 1 else "single GPU",
+                   "launch": launch, "sweep": sweep},
+        "e2e": {"value": ws * nq * args.steps / e2e_s_max, "unit": UNIT,
+                "h2d_bytes_per_step": nq * info.d * 4 + 2 * nq * 4, "d2h_bytes_per_step": 2 * nq * k * 4,
+                "same_ids_as_device_path": e2e_same},
+        "gpu_launches": args.steps,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                     "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": mean_launch_ms,
+                     "kernel": "frog_search_kernel"},
+        "clocks": clocks,
+        "expansions_per_query": float(st[:, 0].mean()), "distances_per_query": float(st[:, 3].mean()),
+        "enc_rows_per_query": float(st[:, 1].mean()),
+    }
+    if cpu:
+        out["cpu_baseline"] = cpu
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="sift")
+    ap.add_argument("--n", type=int, default=0, help="override the number of base vectors (profiling on a small case)")
+    ap.add_argument("--nq", type=int, default=0, help="override the number of queries")
+    ap.add_argument("--beam", type=int, default=0, help="beam width; 0 = smallest reaching the recall target")
+    ap.add_argument("--cache-dir", default=os.environ.get("FROG_CACHE", "/tmp/frog_cache"))
+    ap.add_argument("--cpu-sample", type=int, default=4000)
+    ap.add_argument("--ref-sample", type=int, default=1000)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    ensure_built()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

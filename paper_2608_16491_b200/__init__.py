@@ -20,7 +20,7 @@ from typing import Optional
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_SEARCH = os.path.join(_HERE, "libfrog.so")
+_LIB_SEARCH = os.environ.get("FROG_LIBFROG", os.path.join(_HERE, "libfrog.so"))   # override: A/B builds
 _LIB_BUILD = os.path.join(_HERE, "libfrog_build.so")
 
 FROG_MAX_BEAM_WIDTH = 512

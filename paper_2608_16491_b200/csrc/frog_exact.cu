@@ -34,8 +34,7 @@ frog_exact_kernel(const ExactArgs A) {
     const int q = blockIdx.x;
     float4* qs = reinterpret_cast<float4*>(smem_raw);
     uint64_t* pools = reinterpret_cast<uint64_t*>(smem_raw + (size_t)A.d_pad * 4);
-    uint64_t* pool = pools + (size_t)warp * (POOL + 32);
-    uint64_t* nk = pool + POOL;
+    uint64_t* pool = pools + (size_t)warp * POOL;
 
     {
         float* qf = reinterpret_cast<float*>(qs);
@@ -44,28 +43,26 @@ frog_exact_kernel(const ExactArgs A) {
         for (int i = lane; i < POOL; i += 32) pool[i] = KEY_EMPTY;
     }
     const int32_t lo = __ldg(A.lo + q), hi = __ldg(A.hi + q);
-    const int l_q = warp_count_below(A.sorted_attr, A.n, lo, false, lane);
-    const int r_q = warp_count_below(A.sorted_attr, A.n, hi, true, lane) - 1;
+    int l_q, r_q;
+    warp_rank_interval(A.sorted_attr, A.n, lo, hi, lane, l_q, r_q);
     const int w = (lo > hi) ? 0 : (r_q - l_q + 1);
     __syncthreads();
 
     for (int b0 = warp * 16; b0 < w; b0 += EXACT_WARPS * 16) {
         const int cnt = min(16, w - b0);
         const uint32_t rank = (uint32_t)(l_q + b0 + (lane & 15));
-        float d2 = batch_dist2(A.vectors, A.d_pad, qs, rank, cnt, lane);
+        float d2 = batch_dist2<2>(A.vectors, A.d_pad, qs, rank, cnt, lane);
         uint64_t key = lane < cnt ? make_key(d2, rank, 1u) : KEY_EMPTY;
-        // candidates not better than the current k-th best cannot enter
-        const uint64_t worst = pool[A.k - 1];
-        if (key != KEY_EMPTY && worst != KEY_EMPTY && (key >> 1) >= (worst >> 1)) key = KEY_EMPTY;
-        if (__any_sync(FULL, key != KEY_EMPTY)) merge_batch<EPL>(pool, nk, key, A.k, lane);
+        // (merge_batch itself rejects candidates not better than the current k-th best)
+        merge_batch<EPL>(pool, key, A.k, lane);
     }
     __syncthreads();
     if (warp == 0) {
         for (int ow = 1; ow < EXACT_WARPS; ++ow) {
-            const uint64_t* other = pools + (size_t)ow * (POOL + 32);
+            const uint64_t* other = pools + (size_t)ow * POOL;
             for (int j0 = 0; j0 < A.k; j0 += 32) {
                 uint64_t key = (j0 + lane < A.k) ? other[j0 + lane] : KEY_EMPTY;
-                if (__any_sync(FULL, key != KEY_EMPTY)) merge_batch<EPL>(pool, nk, key, A.k, lane);
+                merge_batch<EPL>(pool, key, A.k, lane);
             }
         }
         __syncwarp();
@@ -101,7 +98,7 @@ extern "C" int frog_exact_search(const frog_index_t* index, const float* queries
     else if (k <= 128) { fn = frog_exact_kernel<4>; pool_slots = 128; }
     else if (k <= 256) { fn = frog_exact_kernel<8>; pool_slots = 256; }
     else { fn = frog_exact_kernel<16>; pool_slots = 512; }
-    size_t smem = (size_t)index->info.d_pad * 4 + (size_t)EXACT_WARPS * (pool_slots + 32) * 8;
+    size_t smem = (size_t)index->info.d_pad * 4 + (size_t)EXACT_WARPS * pool_slots * 8;
     FROG_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     ExactArgs A;
     A.sorted_attr = index->d_sorted_attr;

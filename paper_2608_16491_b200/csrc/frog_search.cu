@@ -17,17 +17,24 @@ using namespace frogdev;
 namespace {
 
 constexpr int WARPS_PER_CTA = 4;
+#ifndef FROG_MINB
+#define FROG_MINB 4
+#endif
+#ifndef FROG_NG
+#define FROG_NG 2
+#endif
+
+constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2;
 
 struct WarpSmem {
     uint64_t* pool;
-    uint64_t* nk;
-    uint32_t* en;
+    uint32_t* cand;
     float4* q;
     uint32_t* hash;
 };
 
 __host__ __device__ inline size_t warp_smem_bytes(int pool_slots, int d_pad, int hash_bits) {
-    return (size_t)pool_slots * 8 + 32 * 8 + 32 * 4 + (size_t)d_pad * 4 + ((size_t)4 << hash_bits);
+    return (size_t)pool_slots * 8 + 32 * 4 + (size_t)d_pad * 4 + ((size_t)4 << hash_bits);
 }
 
 // entry point j of a query range: stateless mixer of (seed, l_q, r_q, j), top 32 bits scaled
@@ -43,42 +50,27 @@ __device__ __forceinline__ uint32_t entry_point(unsigned long long seed, uint32_
     return l_q + (uint32_t)(((x >> 32) * w) >> 32);
 }
 
-// One batch of up to 32 candidate ranks (lane j < cnt holds cand): drop repeats inside the batch,
-// apply the visited check, compute the distances of the survivors, merge them into the pool.
-// Returns the first unexpanded pool position.
+// Distances of the ns ranks listed in S.cand[0..ns) and their merge into the pool (Alg. 2 lines
+// 14-17).  Returns the first unexpanded pool position.
 template <int EPL>
-__device__ __forceinline__ int evaluate_batch(const FrogSearchArgs& A, const WarpSmem& S, uint32_t cand,
-                                              int cnt, bool use_hash, uint32_t new_flag, int lane,
-                                              uint32_t& n_dist, uint32_t& forgets) {
-    bool keep = lane < cnt;
-    if (use_hash) {
-        // the same vertex can sit in several layers of ENC(u): keep its first copy only
-        uint32_t same = __match_any_sync(FULL, keep ? cand : (0x80000000u | (uint32_t)lane));
-        keep = keep && ((__ffs(same) - 1) == lane);
-        if (keep) keep = visited_insert(S.hash, A.hash_bits, cand, forgets);
-    }
-    // compact the survivors to lanes 0..ns-1
-    uint32_t M = __ballot_sync(FULL, keep);
-    int ns = __popc(M);
-    __syncwarp();
-    if (keep) S.en[__popc(M & ((1u << lane) - 1u))] = cand;
-    __syncwarp();
-    uint32_t id = lane < ns ? S.en[lane] : 0u;
-    __syncwarp();
-    n_dist += ns;
+__device__ __forceinline__ int evaluate_and_merge(const FrogSearchArgs& A, const WarpSmem& S, int ns,
+                                                  uint32_t new_flag, int lane) {
     int first = NO_POS;
-    for (int base = 0; base < max(ns, 1); base += 16) {
-        uint32_t sub_id = __shfl_sync(FULL, id, (base + lane) & 31);
-        int sub_ns = min(16, ns - base);
-        float d2 = sub_ns > 0 ? batch_dist2(A.vectors, A.d_pad, S.q, sub_id, sub_ns, lane) : 0.f;
-        uint64_t key = (lane < sub_ns) ? make_key(d2, sub_id, new_flag) : KEY_EMPTY;
-        first = merge_batch<EPL>(S.pool, S.nk, key, A.ef_s, lane);
-    }
+    int base = 0;
+    do {
+        const int sub_ns = min(16, ns - base);
+        const uint32_t id = (lane < sub_ns) ? S.cand[base + lane] : 0u;
+        float d2 = 0.f;
+        if (sub_ns > 0) d2 = batch_dist2<FROG_NG>(A.vectors, A.d_pad, S.q, id, sub_ns, lane);
+        const uint64_t key = (lane < sub_ns) ? make_key(d2, id, new_flag) : KEY_EMPTY;
+        first = merge_batch<EPL>(S.pool, key, A.ef_s, lane);
+        base += 16;
+    } while (base < ns);
     return first;
 }
 
-template <int EPL, bool TRACE>
-__global__ void __launch_bounds__(WARPS_PER_CTA * 32)
+template <int EPL, int MODE>
+__global__ void __launch_bounds__(WARPS_PER_CTA * 32, MODE == MODE_FAST ? (EPL <= 4 ? FROG_MINB : 2) : 1)
 frog_search_kernel(const FrogSearchArgs A) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int lane = lane_id();
@@ -88,17 +80,28 @@ frog_search_kernel(const FrogSearchArgs A) {
     unsigned char* base = smem_raw + per_warp * warp;
     WarpSmem S;
     S.pool = reinterpret_cast<uint64_t*>(base);
-    S.nk = S.pool + POOL;
-    S.en = reinterpret_cast<uint32_t*>(S.nk + 32);
-    S.q = reinterpret_cast<float4*>(S.en + 32);
+    S.cand = reinterpret_cast<uint32_t*>(S.pool + POOL);
+    S.q = reinterpret_cast<float4*>(S.cand + 32);
     S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<float*>(S.q) + A.d_pad);
     const int hash_slots = 1 << A.hash_bits;
+    const uint32_t lt_mask = (1u << lane) - 1u;
 
     for (;;) {
         int q = 0;
         if (lane == 0) q = (int)atomicAdd(A.work_counter, 1u);
         q = __shfl_sync(FULL, q, 0);
         if (q >= A.nq) break;
+
+        long long t_ph[5] = {0, 0, 0, 0, 0};   // set-up, ENC scan, visited check, gather+distance+merge, output
+        long long t_mark = (MODE == MODE_PROFILE) ? clock64() : 0;
+#define FROG_PHASE(i)                                                        \
+    do {                                                                     \
+        if (MODE == MODE_PROFILE) {                                          \
+            long long _n = clock64();                                        \
+            t_ph[i] += _n - t_mark;                                          \
+            t_mark = _n;                                                     \
+        }                                                                    \
+    } while (0)
 
         // ---- per-query set-up ---------------------------------------------------------------
         {
@@ -108,14 +111,13 @@ frog_search_kernel(const FrogSearchArgs A) {
             for (int i = lane; i < POOL; i += 32) S.pool[i] = KEY_EMPTY;
         }
         const int32_t lo = __ldg(A.lo + q), hi = __ldg(A.hi + q);
-        // Sec. 4: [lo, hi] -> rank interval [l_q, r_q]
-        const int l_q = warp_count_below(A.sorted_attr, A.n, lo, false, lane);
-        const int r_q = warp_count_below(A.sorted_attr, A.n, hi, true, lane) - 1;
+        int l_q, r_q;
+        warp_rank_interval(A.sorted_attr, A.n, lo, hi, lane, l_q, r_q);    // Sec. 4
         const int w = (lo > hi) ? 0 : (r_q - l_q + 1);
         uint32_t st = 0, n_exp = 0, n_rows = 0, n_en = 0, n_dist = 0, forgets = 0;
         uint32_t trace_len = 0;
         bool trace_ok = true;
-        uint32_t* trace_row = TRACE ? A.trace + (size_t)q * A.trace_cap : nullptr;
+        uint32_t* trace_row = (MODE != MODE_FAST) ? A.trace + (size_t)q * A.trace_cap : nullptr;
         __syncwarp();
 
         if (w <= 0) {
@@ -124,8 +126,12 @@ frog_search_kernel(const FrogSearchArgs A) {
             // every valid object enters the pool: exact answer
             st |= FROG_ST_EXACT;
             for (int b0 = 0; b0 < w; b0 += 32) {
-                int cnt = min(32, w - b0);
-                evaluate_batch<EPL>(A, S, (uint32_t)(l_q + b0 + lane), cnt, false, 1u, lane, n_dist, forgets);
+                const int cnt = min(32, w - b0);
+                if (lane < cnt) S.cand[lane] = (uint32_t)(l_q + b0 + lane);
+                __syncwarp();
+                evaluate_and_merge<EPL>(A, S, cnt, 1u, lane);
+                n_dist += cnt;
+                __syncwarp();
             }
         } else {
             {
@@ -139,34 +145,79 @@ frog_search_kernel(const FrogSearchArgs A) {
             const int total = (L_end - L_start + 1) * A.m;
             const uint32_t span = (uint32_t)(r_q - l_q);
             __syncwarp();
-            // lines 2-5: entry points
-            uint32_t ep = lane < A.epn ? entry_point(A.seed, (uint32_t)l_q, (uint32_t)r_q, lane) : 0u;
-            int first = evaluate_batch<EPL>(A, S, ep, A.epn, true, 0u, lane, n_dist, forgets);
+            // lines 2-5: entry points, passed through the visited set
+            int ns;
+            {
+                const uint32_t ep = entry_point(A.seed, (uint32_t)l_q, (uint32_t)r_q, lane);
+                bool keep = lane < A.epn;
+                if (keep) keep = visited_insert(S.hash, A.hash_bits, ep, forgets);
+                const uint32_t M = __ballot_sync(FULL, keep);
+                if (keep) S.cand[__popc(M & lt_mask)] = ep;
+                ns = __popc(M);
+                __syncwarp();
+            }
+            FROG_PHASE(0);
+            n_dist += ns;
+            int first = evaluate_and_merge<EPL>(A, S, ns, 0u, lane);
+            FROG_PHASE(3);
             // lines 7-17
             while (first < A.ef_s) {
                 if ((int)n_exp >= A.max_iters) { st |= FROG_ST_ITER_CAP; break; }
                 const uint32_t u = key_rank(S.pool[first]);               // line 8
                 __syncwarp();
                 if (lane == 0) S.pool[first] |= 1ull;                     // line 9
+                // line 10, Alg. 4: scan rows L_start..L_end of ENC(u) in 32-entry chunks (two
+                // fetched per round trip); predicate "not empty and l_q <= v <= r_q" as one
+                // unsigned compare (the empty entry 0xFFFFFFFF minus l_q exceeds any span);
+                // ballot + popc give the admitted prefix under budget B.  Lines 12-13: each
+                // admitted lane applies the visited check where it stands; survivors are
+                // compacted into S.cand.
                 const uint32_t* hot = A.enc + ((size_t)u * A.H + L_start) * A.m;
-                int scanned;
-                int cnt = en_identify(hot, total, (uint32_t)l_q, span, A.B, S.en, lane, scanned);   // line 10
+                int cnt = 0, scanned = 0;
+                ns = 0;
+                for (int c0 = 0; c0 < total && cnt < A.B; c0 += 64) {
+                    uint32_t v0 = BOT, v1 = BOT;
+                    if (c0 + lane < total) v0 = ldg_stream_u32(hot + c0 + lane);
+                    if (c0 + 32 + lane < total) v1 = ldg_stream_u32(hot + c0 + 32 + lane);
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        if (half == 1 && (cnt >= A.B || c0 + 32 >= total)) break;
+                        const uint32_t v = half ? v1 : v0;
+                        const bool pred = (v - (uint32_t)l_q) <= span;
+                        const uint32_t M = __ballot_sync(FULL, pred);
+                        const int a = min(__popc(M), A.B - cnt);
+                        const bool admitted = pred && (__popc(M & lt_mask) < a);
+                        if (MODE == MODE_TRACE) {
+                            if (trace_ok && admitted && 3 + trace_len + cnt + 16 < (uint32_t)A.trace_cap)
+                                trace_row[3 + trace_len + cnt + __popc(M & lt_mask)] = v;
+                        }
+                        FROG_PHASE(1);
+                        bool keep = admitted;
+                        if (keep) keep = visited_insert(S.hash, A.hash_bits, v, forgets);
+                        const uint32_t K = __ballot_sync(FULL, keep);
+                        if (keep) S.cand[ns + __popc(K & lt_mask)] = v;
+                        ns += __popc(K);
+                        cnt += a;
+                        scanned = min(total, c0 + 32 * (half + 1));
+                        FROG_PHASE(2);
+                    }
+                }
                 __syncwarp();
-                uint32_t cand = lane < cnt ? S.en[lane] : 0u;
                 ++n_exp;
                 n_rows += (scanned + A.m - 1) / A.m;
                 n_en += cnt;
-                if (TRACE) {
+                n_dist += ns;
+                if (MODE == MODE_TRACE) {
                     // records are appended until the first one that does not fit
                     if (trace_ok && trace_len + 2 + cnt <= (uint32_t)A.trace_cap - 1) {
                         if (lane == 0) { trace_row[1 + trace_len] = u; trace_row[2 + trace_len] = (uint32_t)cnt; }
-                        if (lane < cnt) trace_row[3 + trace_len + lane] = cand;
                         trace_len += 2 + cnt;
                     } else {
                         trace_ok = false;
                     }
                 }
-                first = evaluate_batch<EPL>(A, S, cand, cnt, true, 0u, lane, n_dist, forgets);   // lines 11-17
+                first = evaluate_and_merge<EPL>(A, S, ns, 0u, lane);      // lines 14-17
+                FROG_PHASE(3);
             }
         }
 
@@ -188,28 +239,34 @@ frog_search_kernel(const FrogSearchArgs A) {
         got = __reduce_add_sync(FULL, got);
         if (got < A.k) st |= FROG_ST_SHORT;
         if (__any_sync(FULL, forgets != 0)) st |= FROG_ST_FORGOT;   // counted per lane
+        FROG_PHASE(4);
         if (lane == 0) {
             if (A.status) A.status[q] = st;
             if (A.stats) {
                 uint32_t* srow = A.stats + 4 * (size_t)q;
                 srow[0] = n_exp; srow[1] = n_rows; srow[2] = n_en; srow[3] = n_dist;
             }
-            if (TRACE) trace_row[0] = trace_len;
+            if (MODE == MODE_TRACE) trace_row[0] = trace_len;
+            if (MODE == MODE_PROFILE) {
+                trace_row[0] = 5;
+                for (int i = 0; i < 5; ++i) trace_row[1 + i] = (uint32_t)min(t_ph[i], 0xFFFFFFFFll);
+            }
         }
         __syncwarp();
+#undef FROG_PHASE
     }
 }
 
 typedef void (*kernel_fn)(const FrogSearchArgs);
 
-template <bool TRACE>
+template <int MODE>
 kernel_fn pick_kernel(int ef_s, int* pool_slots) {
-    if (ef_s <= 32) { *pool_slots = 32; return frog_search_kernel<1, TRACE>; }
-    if (ef_s <= 64) { *pool_slots = 64; return frog_search_kernel<2, TRACE>; }
-    if (ef_s <= 128) { *pool_slots = 128; return frog_search_kernel<4, TRACE>; }
-    if (ef_s <= 256) { *pool_slots = 256; return frog_search_kernel<8, TRACE>; }
+    if (ef_s <= 32) { *pool_slots = 32; return frog_search_kernel<1, MODE>; }
+    if (ef_s <= 64) { *pool_slots = 64; return frog_search_kernel<2, MODE>; }
+    if (ef_s <= 128) { *pool_slots = 128; return frog_search_kernel<4, MODE>; }
+    if (ef_s <= 256) { *pool_slots = 256; return frog_search_kernel<8, MODE>; }
     *pool_slots = 512;
-    return frog_search_kernel<16, TRACE>;
+    return frog_search_kernel<16, MODE>;
 }
 
 struct LaunchPlan {
@@ -218,9 +275,11 @@ struct LaunchPlan {
     size_t smem;
 };
 
-int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, bool trace, int nq, LaunchPlan* out) {
+int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, int mode, int nq, LaunchPlan* out) {
     int pool_slots = 0;
-    kernel_fn fn = trace ? pick_kernel<true>(beam_width, &pool_slots) : pick_kernel<false>(beam_width, &pool_slots);
+    kernel_fn fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE>(beam_width, &pool_slots)
+                 : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE>(beam_width, &pool_slots)
+                                        : pick_kernel<MODE_FAST>(beam_width, &pool_slots);
     size_t smem = warp_smem_bytes(pool_slots, ix->info.d_pad, P.hash_bits) * WARPS_PER_CTA;
     if (smem > 227 * 1024) return FROG_ERR_UNSUPPORTED;
     FROG_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -276,7 +335,7 @@ extern "C" int frog_search_launch_info(const frog_index_t* index, int beam_width
     if (rc) return rc;
     FROG_CUDA_TRY(cudaSetDevice(index->info.device));
     LaunchPlan plan;
-    rc = plan_launch(index, beam_width, P, false, 0, &plan);
+    rc = plan_launch(index, beam_width, P, MODE_FAST, 0, &plan);
     if (rc) return rc;
     if (grid) *grid = plan.grid;
     if (block) *block = plan.block;
@@ -291,7 +350,7 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
                               uint32_t* trace, int trace_cap, void* stream) {
     if (!index || nq < 0) return FROG_ERR_INVALID_ARG;
     if (k < 1 || beam_width < 1 || beam_width > FROG_MAX_BEAM_WIDTH || k > beam_width) return FROG_ERR_INVALID_ARG;
-    if (trace && trace_cap < 4) return FROG_ERR_INVALID_ARG;
+    if (trace && trace_cap < 8) return FROG_ERR_INVALID_ARG;
     if (nq == 0) return FROG_OK;
     if (!queries || !lo || !hi || !out_ids || !out_dists) return FROG_ERR_INVALID_ARG;
     frog_params_t P;
@@ -299,7 +358,8 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     if (rc) return rc;
     FROG_CUDA_TRY(cudaSetDevice(index->info.device));
     LaunchPlan plan;
-    rc = plan_launch(index, beam_width, P, trace != nullptr, nq, &plan);
+    const int mode = !trace ? MODE_FAST : (P.reserved & 1) ? MODE_PROFILE : MODE_TRACE;
+    rc = plan_launch(index, beam_width, P, mode, nq, &plan);
     if (rc) return rc;
 
     FrogSearchArgs A;

@@ -75,7 +75,7 @@ def test_tiny_matches_oracle_at_every_beam_width(libs, tiny_gpu, ef):
     wl, ix, gix = tiny_gpu
     ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, ef, trace_cap=40000 if ef <= 128 else 0)
     got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, wl.k, ef, trace_cap=40000 if ef <= 128 else 0)
-    _assert_parity(got, ref)
+    _assert_parity(got, ref, slots=_default_slots(ef))
 
 
 def test_tiny_plain_call_equals_ex_call(libs, tiny_gpu):
@@ -97,7 +97,7 @@ def test_tiny_parameter_variants(libs, tiny_gpu, params):
                no_hotspot=bool(params.get("no_hotspot", 0)), max_iters=params.get("max_iters", 0))
     ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 48, trace_cap=20000, **okw)
     got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, wl.k, 48, trace_cap=20000, **params)
-    _assert_parity(got, ref)
+    _assert_parity(got, ref, slots=_default_slots(48))
 
 
 def test_k_equals_beam_and_k_one(libs, tiny_gpu):
@@ -105,7 +105,7 @@ def test_k_equals_beam_and_k_one(libs, tiny_gpu):
     for k, ef in ((32, 32), (1, 16), (100, 128), (64, 64)):
         ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef)
         got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, k, ef)
-        _assert_parity(got, ref)
+        _assert_parity(got, ref, slots=_default_slots(ef))
 
 
 def test_edge_ranges(libs, tiny_gpu):
