@@ -64,9 +64,19 @@ typedef struct {
     int32_t max_iters;  /* hard cap on expansions per query; 0 = default 16 * beam_width */
     int32_t no_hotspot; /* nonzero: scan all H layers instead of the hotspot (ablation) */
     uint64_t seed;      /* seed of the entry-point generator */
-    int32_t hash_bits;  /* log2 of the per-query visited-table slots; 0 = chosen from beam_width */
+    int32_t hash_bits;  /* FROG_VISITED_HASH: log2 of the table slots; 0 = chosen from beam_width */
+    int32_t visited;    /* FROG_VISITED_*: where the visited set lives */
+    int32_t debug_flags;/* bit 0: with `trace`, record per-phase cycle counts instead of EN lists */
     int32_t reserved;
 } frog_params_t;
+
+/* Visited set (hashCheck of Alg. 2).  BITMAP: one bit per rank in a per-warp slab of device
+ * scratch memory owned by the index (n/8 bytes per resident warp, allocated on first use, exact).
+ * HASH: a bounded table in shared memory, no scratch; a crowded table drops entries, which repeats
+ * distance evaluations but never changes results.  AUTO = BITMAP, HASH if the slabs do not fit. */
+#define FROG_VISITED_AUTO 0
+#define FROG_VISITED_BITMAP 1
+#define FROG_VISITED_HASH 2
 
 /* Per-query status bits written by frog_search_ex. */
 #define FROG_ST_EMPTY 1u     /* lo > hi or no object in [lo, hi]: row is all padding */
@@ -103,8 +113,10 @@ int frog_index_info(const frog_index_t* index, frog_index_info_t* out);
  *   out_dists  DEVICE, nq x k fp32: L2 distances (not squared), ascending; +inf padding
  *   stream     cudaStream_t (as void*); the call only enqueues work and returns
  * The caller owns all buffers and keeps them alive until the stream reaches the end of the
- * call.  Calls on the same index must not overlap on the GPU (they share the index's small
- * scratch: a work counter); serialise them on one stream or with events.  nq == 0 is a no-op.
+ * call.  Calls on the same index must not overlap on the GPU (they share the index's scratch:
+ * a work counter and the visited slabs); serialise them on one stream or with events.  The
+ * first call (and any call that needs more resident warps than all calls before it) allocates
+ * the visited slabs with cudaMalloc after a device synchronise.  nq == 0 is a no-op.
  * Errors: INVALID_ARG, UNSUPPORTED, CUDA (launch failure).  Per-query conditions (empty range,
  * iteration cap, fewer than k results) are not errors; see frog_search_ex. */
 int frog_search(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
@@ -116,9 +128,8 @@ int frog_search(const frog_index_t* index, const float* queries, const int32_t* 
  *   stats   DEVICE nq x 4 uint32 or null: {expansions, ENC rows the scan needed, ENs admitted
  *           by Alg. 4, distance evaluations}
  *   trace   DEVICE nq x trace_cap uint32 or null: row q = [len, then per expansion
- *           u, |EN(u)|, EN(u)[0..]] (ranks), records appended until the first that would
- *           exceed trace_cap-1 words.  Selects a
- *           slower kernel instantiation; meant for tests. */
+ *           u, |EN(u)|, EN(u)[0..]] (ranks); records are appended while at least 66 words
+ *           remain in the row.  Selects a slower kernel instantiation; meant for tests. */
 int frog_search_ex(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
                    int nq, int k, int beam_width, const frog_params_t* params,
                    int32_t* out_ids, float* out_dists, uint32_t* status, uint32_t* stats,
@@ -136,7 +147,8 @@ int frog_exact_search(const frog_index_t* index, const float* queries, const int
  * the copies asynchronous); copies in, searches, copies the results out and synchronises the
  * stream.  Uses staging buffers owned by the index, grown on first use. */
 int frog_search_host(frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
-                     int nq, int k, int beam_width, int32_t* out_ids, float* out_dists, void* stream);
+                     int nq, int k, int beam_width, const frog_params_t* params /* HOST, may be null */,
+                     int32_t* out_ids, float* out_dists, void* stream);
 
 /* Launch shape of the search kernel for the given beam width (for reporting): CTAs, threads per
  * CTA, dynamic shared memory per CTA, query slots resident per SM. */

@@ -25,6 +25,7 @@ _LIB_BUILD = os.path.join(_HERE, "libfrog_build.so")
 
 FROG_MAX_BEAM_WIDTH = 512
 ST_EMPTY, ST_EXACT, ST_ITER_CAP, ST_SHORT, ST_FORGOT = 1, 2, 4, 8, 16
+VISITED_AUTO, VISITED_BITMAP, VISITED_HASH = 0, 1, 2
 
 
 class FrogError(RuntimeError):
@@ -43,7 +44,7 @@ class IndexInfo(C.Structure):
 class Params(C.Structure):
     _fields_ = [("epn", C.c_int32), ("budget", C.c_int32), ("max_iters", C.c_int32),
                 ("no_hotspot", C.c_int32), ("seed", C.c_uint64), ("hash_bits", C.c_int32),
-                ("reserved", C.c_int32)]
+                ("visited", C.c_int32), ("debug_flags", C.c_int32), ("reserved", C.c_int32)]
 
 
 class BuildParams(C.Structure):
@@ -203,7 +204,7 @@ class Index:
 
     # -- host buffers in, host buffers out (transfers inside the call) ---------------------------
     def search_host(self, queries, lo, hi, k: int, beam_width: int, out_ids=None, out_dists=None,
-                    stream=None):
+                    stream=None, params: Optional[Params] = None):
         """queries/lo/hi: CPU torch tensors or numpy arrays (pinned memory makes copies async)."""
         import torch
         tq, tlo, thi = (torch.as_tensor(x) for x in (queries, lo, hi))
@@ -215,7 +216,8 @@ class Index:
         if out_dists is None:
             out_dists = torch.empty((nq, k), dtype=torch.float32).pin_memory()
         rc = _lib.frog_search_host(self._h, _ptr(tq), _ptr(tlo), _ptr(thi), C.c_int(nq), C.c_int(k),
-                                   C.c_int(beam_width), _ptr(out_ids), _ptr(out_dists), _stream_ptr(stream))
+                                   C.c_int(beam_width), C.byref(params) if params is not None else None,
+                                   _ptr(out_ids), _ptr(out_dists), _stream_ptr(stream))
         if rc:
             raise FrogError(rc, "frog_search_host")
         return out_ids, out_dists

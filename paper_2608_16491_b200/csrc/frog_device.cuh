@@ -133,63 +133,68 @@ __device__ __forceinline__ bool visited_insert(uint32_t* tab, int bits, uint32_t
 // increasing g with acc = fma(x - q, x - q, acc) element by element; then the 8 partial sums are
 // combined by xor-butterfly with partner distance 4, 2, 1.
 // Memory: the four teams of a warp fetch four different rows per instruction, each team reading
-// 128 contiguous bytes (8 x 16-byte loads) -- whole 32-byte sectors only.  NG loads per row are in
-// flight per lane (NG * 4 in total when all four rounds are live).
+// 128 contiguous bytes (8 x 16-byte loads) -- whole 32-byte sectors only.  Rows are taken two
+// rounds (8 rows) at a time with NG groups of each in flight per lane: for d <= 32*NG all loads
+// of up to 8 rows are issued before the first use, i.e. one memory round trip.
 template <int NG>
 __device__ __forceinline__ float batch_dist2(const float* __restrict__ vectors, int d_pad,
                                              const float4* qs, uint32_t my_rank, int ns, int lane) {
     const int team = lane >> 3, sub = lane & 7;
     const int G = d_pad >> 2;
-    const int rounds = (ns + 3) >> 2;
-    const float4* row[4];
-    bool valid[4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        int vi = r * 4 + team;
-        uint32_t id = __shfl_sync(FULL, my_rank, vi);
-        valid[r] = vi < ns;
-        row[r] = reinterpret_cast<const float4*>(vectors + (size_t)id * (size_t)d_pad);
-    }
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float out = 0.f;
+    const int src = (lane & 3) << 3;
 #pragma unroll 1
-    for (int g0 = sub; g0 < G; g0 += 8 * NG) {
-        float4 x[4][NG];
+    for (int r0 = 0; r0 * 4 < ns; r0 += 2) {
+        const int viA = r0 * 4 + team, viB = viA + 4;
+        const bool vA = viA < ns, vB = viB < ns;
+        const bool anyB = (r0 + 1) * 4 < ns;                    // warp-uniform
+        const uint32_t idA = __shfl_sync(FULL, my_rank, viA & 31);
+        const uint32_t idB = __shfl_sync(FULL, my_rank, viB & 31);
+        const float4* rowA = reinterpret_cast<const float4*>(vectors + (size_t)idA * (size_t)d_pad) + sub;
+        const float4* rowB = reinterpret_cast<const float4*>(vectors + (size_t)idB * (size_t)d_pad) + sub;
+        float accA = 0.f, accB = 0.f;
+#pragma unroll 1
+        for (int g0 = sub; g0 < G; g0 += 8 * NG) {
+            float4 xa[NG], xb[NG];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            if (r < rounds && valid[r]) {
-#pragma unroll
-                for (int c = 0; c < NG; ++c)
-                    if (c == 0 || g0 + 8 * c < G) x[r][c] = ldg_stream_f4(row[r] + g0 + 8 * c);
+            for (int c = 0; c < NG; ++c) {
+                if (g0 + 8 * c < G) {
+                    if (vA) xa[c] = ldg_stream_f4(rowA + (g0 - sub) + 8 * c);
+                    if (vB) xb[c] = ldg_stream_f4(rowB + (g0 - sub) + 8 * c);
+                }
             }
-        }
 #pragma unroll
-        for (int c = 0; c < NG; ++c) {
-            if (c == 0 || g0 + 8 * c < G) {
-                const float4 q = qs[g0 + 8 * c];
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    if (r < rounds && valid[r]) {
-                        float t;
-                        t = x[r][c].x - q.x; acc[r] = fmaf(t, t, acc[r]);
-                        t = x[r][c].y - q.y; acc[r] = fmaf(t, t, acc[r]);
-                        t = x[r][c].z - q.z; acc[r] = fmaf(t, t, acc[r]);
-                        t = x[r][c].w - q.w; acc[r] = fmaf(t, t, acc[r]);
+            for (int c = 0; c < NG; ++c) {
+                if (g0 + 8 * c < G) {
+                    const float4 q = qs[g0 + 8 * c];
+                    float t;
+                    if (vA) {
+                        t = xa[c].x - q.x; accA = fmaf(t, t, accA);
+                        t = xa[c].y - q.y; accA = fmaf(t, t, accA);
+                        t = xa[c].z - q.z; accA = fmaf(t, t, accA);
+                        t = xa[c].w - q.w; accA = fmaf(t, t, accA);
+                    }
+                    if (vB) {
+                        t = xb[c].x - q.x; accB = fmaf(t, t, accB);
+                        t = xb[c].y - q.y; accB = fmaf(t, t, accB);
+                        t = xb[c].z - q.z; accB = fmaf(t, t, accB);
+                        t = xb[c].w - q.w; accB = fmaf(t, t, accB);
                     }
                 }
             }
         }
-    }
-    // row j was handled by team j & 3 in round j >> 2
-    float out = 0.f;
-    const int src = (lane & 3) << 3;
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        if (r < rounds) {
-            acc[r] = acc[r] + __shfl_xor_sync(FULL, acc[r], 4);
-            acc[r] = acc[r] + __shfl_xor_sync(FULL, acc[r], 2);
-            acc[r] = acc[r] + __shfl_xor_sync(FULL, acc[r], 1);
-            float v = __shfl_sync(FULL, acc[r], src);
-            if ((lane >> 2) == r) out = v;
+        // row j was handled by team j & 3 in round j >> 2
+        accA = accA + __shfl_xor_sync(FULL, accA, 4);
+        accA = accA + __shfl_xor_sync(FULL, accA, 2);
+        accA = accA + __shfl_xor_sync(FULL, accA, 1);
+        const float va = __shfl_sync(FULL, accA, src);
+        if ((lane >> 2) == r0) out = va;
+        if (anyB) {
+            accB = accB + __shfl_xor_sync(FULL, accB, 4);
+            accB = accB + __shfl_xor_sync(FULL, accB, 2);
+            accB = accB + __shfl_xor_sync(FULL, accB, 1);
+            const float vb = __shfl_sync(FULL, accB, src);
+            if ((lane >> 2) == r0 + 1) out = vb;
         }
     }
     return out;

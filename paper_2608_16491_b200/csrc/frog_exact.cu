@@ -51,7 +51,7 @@ frog_exact_kernel(const ExactArgs A) {
     for (int b0 = warp * 16; b0 < w; b0 += EXACT_WARPS * 16) {
         const int cnt = min(16, w - b0);
         const uint32_t rank = (uint32_t)(l_q + b0 + (lane & 15));
-        float d2 = batch_dist2<2>(A.vectors, A.d_pad, qs, rank, cnt, lane);
+        float d2 = batch_dist2<4>(A.vectors, A.d_pad, qs, rank, cnt, lane);
         uint64_t key = lane < cnt ? make_key(d2, rank, 1u) : KEY_EMPTY;
         // (merge_batch itself rejects candidates not better than the current k-th best)
         merge_batch<EPL>(pool, key, A.k, lane);

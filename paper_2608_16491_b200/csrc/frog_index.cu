@@ -112,6 +112,7 @@ extern "C" void frog_index_free(frog_index_t* ix) {
         cudaFree(ix->d_vectors);
         cudaFree(ix->d_enc);
         cudaFree(ix->d_work);
+        cudaFree(ix->d_bitmap);
         cudaFree(ix->d_stage);
     }
     delete ix;
@@ -204,7 +205,8 @@ extern "C" int frog_index_from_host(const int32_t* sorted_attr, const int32_t* r
 }
 
 extern "C" int frog_search_host(frog_index_t* ix, const float* queries, const int32_t* lo, const int32_t* hi,
-                                int nq, int k, int beam_width, int32_t* out_ids, float* out_dists, void* stream) {
+                                int nq, int k, int beam_width, const frog_params_t* params,
+                                int32_t* out_ids, float* out_dists, void* stream) {
     if (!ix || nq < 0) return FROG_ERR_INVALID_ARG;
     if (k < 1 || beam_width < 1 || beam_width > FROG_MAX_BEAM_WIDTH || k > beam_width) return FROG_ERR_INVALID_ARG;
     if (nq == 0) return FROG_OK;
@@ -232,7 +234,8 @@ extern "C" int frog_search_host(frog_index_t* ix, const float* queries, const in
     FROG_CUDA_TRY(cudaMemcpyAsync(d_q, queries, (size_t)nq * ix->info.d * 4, cudaMemcpyHostToDevice, s));
     FROG_CUDA_TRY(cudaMemcpyAsync(d_lo, lo, (size_t)nq * 4, cudaMemcpyHostToDevice, s));
     FROG_CUDA_TRY(cudaMemcpyAsync(d_hi, hi, (size_t)nq * 4, cudaMemcpyHostToDevice, s));
-    int rc = frog_search(ix, d_q, d_lo, d_hi, nq, k, beam_width, d_ids, d_dist, stream);
+    int rc = frog_search_ex(ix, d_q, d_lo, d_hi, nq, k, beam_width, params, d_ids, d_dist, nullptr, nullptr,
+                            nullptr, 0, stream);
     if (rc != FROG_OK) return rc;
     FROG_CUDA_TRY(cudaMemcpyAsync(out_ids, d_ids, (size_t)nq * k * 4, cudaMemcpyDeviceToHost, s));
     FROG_CUDA_TRY(cudaMemcpyAsync(out_dists, d_dist, (size_t)nq * k * 4, cudaMemcpyDeviceToHost, s));

@@ -13,6 +13,8 @@ struct frog_index {
     float* d_vectors = nullptr;      // n x d_pad, rank order
     uint32_t* d_enc = nullptr;       // n x H x m
     unsigned int* d_work = nullptr;  // scratch: work counter of the persistent kernel (+ spare words)
+    uint32_t* d_bitmap = nullptr;    // scratch: per-warp visited slabs (bitmap_slots x words per slot)
+    size_t bitmap_slots = 0;
     // staging for frog_search_host, grown on demand
     void* d_stage = nullptr;
     size_t stage_bytes = 0;
@@ -38,11 +40,14 @@ struct FrogSearchArgs {
     uint32_t* trace;
     int trace_cap;
     unsigned int* work_counter;
+    uint32_t* bitmap;          // visited slabs, or null when the shared-memory table is used
+    size_t bitmap_words;       // words per slab
 };
 
 namespace froghost {
 void set_cuda_error(cudaError_t e);
 int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in, frog_params_t* out);
+int ensure_bitmap(const frog_index* ix, size_t slots);
 }  // namespace froghost
 
 #define FROG_CUDA_TRY(expr)                                  \

@@ -2,10 +2,17 @@
 //
 // Mapping.  Queries are independent (Sec. 7.1), so each WARP owns one query at a time and pulls
 // the next one from a global work counter; a CTA is just a bundle of such warps, they never
-// synchronise with each other.  Per-query state lives in that warp's slice of shared memory:
-// the candidate pool (sorted u64 keys), the new-candidate keys, the compacted EN array, the
-// query vector and the visited table.  Global memory holds the ENC array and the vectors; per
-// expansion the warp reads the hotspot rows of ENC(u) and the rows of the surviving ENs only.
+// synchronise with each other.  Per-query state lives in that warp's slice of shared memory: the
+// candidate pool (sorted u64 keys), the compacted candidate list and the query vector.  Global
+// memory holds the ENC array and the vectors; per expansion the warp reads the hotspot rows of
+// ENC(u) and the rows of the surviving ENs only.
+//
+// Visited set (the hashCheck of Alg. 2 line 12), two interchangeable forms:
+//   * BITMAP: one bit per rank in a per-warp slab of global scratch memory, test-and-set with a
+//     single atomicOr (exact, no probing, no shared memory; the warp clears the words covering
+//     [l_q, r_q] when it starts a query; the slab stays L2-resident while the query runs);
+//   * HASH: an open-addressing table in shared memory (no scratch besides the work counter; a
+//     crowded table forgets entries, which costs repeated distance evaluations, never results).
 #include <cstdio>
 #include <cstring>
 
@@ -16,14 +23,17 @@ using namespace frogdev;
 
 namespace {
 
-constexpr int WARPS_PER_CTA = 4;
+constexpr int WARPS_PER_CTA = 2;
 #ifndef FROG_MINB
-#define FROG_MINB 4
+#define FROG_MINB 16          // resident CTAs per SM the register allocation aims at (EPL <= 4)
 #endif
 #ifndef FROG_NG
 #define FROG_NG 2
 #endif
 
+#ifndef FROG_EVAL_INLINE
+#define FROG_EVAL_INLINE __noinline__
+#endif
 constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2;
 
 struct WarpSmem {
@@ -33,8 +43,8 @@ struct WarpSmem {
     uint32_t* hash;
 };
 
-__host__ __device__ inline size_t warp_smem_bytes(int pool_slots, int d_pad, int hash_bits) {
-    return (size_t)pool_slots * 8 + 32 * 4 + (size_t)d_pad * 4 + ((size_t)4 << hash_bits);
+inline size_t warp_smem_bytes(int pool_slots, int d_pad, int hash_bits, bool bitmap) {
+    return (size_t)pool_slots * 8 + 32 * 4 + (size_t)d_pad * 4 + (bitmap ? 0 : ((size_t)4 << hash_bits));
 }
 
 // entry point j of a query range: stateless mixer of (seed, l_q, r_q, j), top 32 bits scaled
@@ -50,40 +60,57 @@ __device__ __forceinline__ uint32_t entry_point(unsigned long long seed, uint32_
     return l_q + (uint32_t)(((x >> 32) * w) >> 32);
 }
 
-// Distances of the ns ranks listed in S.cand[0..ns) and their merge into the pool (Alg. 2 lines
-// 14-17).  Returns the first unexpanded pool position.
-template <int EPL>
-__device__ __forceinline__ int evaluate_and_merge(const FrogSearchArgs& A, const WarpSmem& S, int ns,
-                                                  uint32_t new_flag, int lane) {
-    int first = NO_POS;
-    int base = 0;
-    do {
-        const int sub_ns = min(16, ns - base);
-        const uint32_t id = (lane < sub_ns) ? S.cand[base + lane] : 0u;
-        float d2 = 0.f;
-        if (sub_ns > 0) d2 = batch_dist2<FROG_NG>(A.vectors, A.d_pad, S.q, id, sub_ns, lane);
-        const uint64_t key = (lane < sub_ns) ? make_key(d2, id, new_flag) : KEY_EMPTY;
-        first = merge_batch<EPL>(S.pool, key, A.ef_s, lane);
-        base += 16;
-    } while (base < ns);
-    return first;
+// test-and-set of rank v in the visited set; true iff v had not been evaluated yet
+template <bool BITMAP>
+__device__ __forceinline__ bool visited_test_and_set(const WarpSmem& S, uint32_t* bitmap, int hash_bits,
+                                                     uint32_t v, uint32_t& forgets) {
+    if (BITMAP) {
+        const uint32_t bit = 1u << (v & 31);
+        return (atomicOr(bitmap + (v >> 5), bit) & bit) == 0;
+    } else {
+        return visited_insert(S.hash, hash_bits, v, forgets);
+    }
 }
 
-template <int EPL, int MODE>
-__global__ void __launch_bounds__(WARPS_PER_CTA * 32, MODE == MODE_FAST ? (EPL <= 4 ? FROG_MINB : 2) : 1)
+// Distances of the ns <= 32 ranks listed in cand[0..ns) and their merge into the pool (Alg. 2
+// lines 14-17).  Returns the first unexpanded pool position.  Kept out of line: it is called from
+// three places of the kernel and inlining every copy costs registers and instruction cache.
+template <int EPL>
+__device__ FROG_EVAL_INLINE int evaluate_and_merge(const float* __restrict__ vectors, int d_pad, int ef_s,
+                                                   uint64_t* pool, const uint32_t* cand, const float4* qs,
+                                                   int ns, uint32_t new_flag, long long* t_dist) {
+    const int lane = lane_id();
+    const uint32_t id = (lane < ns) ? cand[lane] : 0u;
+    float d2 = 0.f;
+    if (ns > 0) d2 = batch_dist2<FROG_NG>(vectors, d_pad, qs, id, min(ns, 16), lane);
+    if (ns > 16) {
+        // rows 16..31: computed with the ids moved down to lanes 0..15, result moved back up
+        const uint32_t id_hi = __shfl_down_sync(FULL, id, 16);
+        const float d_hi = batch_dist2<FROG_NG>(vectors, d_pad, qs, id_hi, ns - 16, lane);
+        const float up = __shfl_up_sync(FULL, d_hi, 16);
+        if (lane >= 16) d2 = up;
+    }
+    const uint64_t key = (lane < ns) ? make_key(d2, id, new_flag) : KEY_EMPTY;
+    if (t_dist) *t_dist = clock64();
+    return merge_batch<EPL>(pool, key, ef_s, lane);
+}
+
+template <int EPL, int MODE, bool BITMAP>
+__global__ void __launch_bounds__(WARPS_PER_CTA * 32, MODE == MODE_FAST ? (EPL <= 4 ? FROG_MINB : 4) : 1)
 frog_search_kernel(const FrogSearchArgs A) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int lane = lane_id();
     const int warp = threadIdx.x >> 5;
     constexpr int POOL = 32 * EPL;
-    const size_t per_warp = warp_smem_bytes(POOL, A.d_pad, A.hash_bits);
+    const int hash_slots = BITMAP ? 0 : (1 << A.hash_bits);
+    const size_t per_warp = (size_t)POOL * 8 + 32 * 4 + (size_t)A.d_pad * 4 + (size_t)hash_slots * 4;
     unsigned char* base = smem_raw + per_warp * warp;
     WarpSmem S;
     S.pool = reinterpret_cast<uint64_t*>(base);
     S.cand = reinterpret_cast<uint32_t*>(S.pool + POOL);
     S.q = reinterpret_cast<float4*>(S.cand + 32);
     S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<float*>(S.q) + A.d_pad);
-    const int hash_slots = 1 << A.hash_bits;
+    uint32_t* bitmap = BITMAP ? A.bitmap + (size_t)(blockIdx.x * WARPS_PER_CTA + warp) * A.bitmap_words : nullptr;
     const uint32_t lt_mask = (1u << lane) - 1u;
 
     for (;;) {
@@ -92,9 +119,9 @@ frog_search_kernel(const FrogSearchArgs A) {
         q = __shfl_sync(FULL, q, 0);
         if (q >= A.nq) break;
 
-        long long t_ph[5] = {0, 0, 0, 0, 0};   // set-up, ENC scan, visited check, gather+distance+merge, output
+        long long t_ph[6] = {0, 0, 0, 0, 0, 0};   // set-up, ENC scan, visited check, gather+distance, output, merge
         long long t_mark = (MODE == MODE_PROFILE) ? clock64() : 0;
-#define FROG_PHASE(i)                                                        \
+ #define FROG_PHASE(i)                                                        \
     do {                                                                     \
         if (MODE == MODE_PROFILE) {                                          \
             long long _n = clock64();                                        \
@@ -102,6 +129,20 @@ frog_search_kernel(const FrogSearchArgs A) {
             t_mark = _n;                                                     \
         }                                                                    \
     } while (0)
+
+        // distance + merge call; in profile builds the time is split at the end of the distances
+        long long t_split = 0;
+        auto EVAL = [&](int ns_, uint32_t flag_) {
+            int f_ = evaluate_and_merge<EPL>(A.vectors, A.d_pad, A.ef_s, S.pool, S.cand, S.q, ns_, flag_,
+                                             MODE == MODE_PROFILE ? &t_split : nullptr);
+            if (MODE == MODE_PROFILE) {
+                long long n_ = clock64();
+                t_ph[3] += t_split - t_mark;
+                t_ph[5] += n_ - t_split;
+                t_mark = n_;
+            }
+            return f_;
+        };
 
         // ---- per-query set-up ---------------------------------------------------------------
         {
@@ -129,12 +170,16 @@ frog_search_kernel(const FrogSearchArgs A) {
                 const int cnt = min(32, w - b0);
                 if (lane < cnt) S.cand[lane] = (uint32_t)(l_q + b0 + lane);
                 __syncwarp();
-                evaluate_and_merge<EPL>(A, S, cnt, 1u, lane);
+                EVAL(cnt, 1u);
                 n_dist += cnt;
                 __syncwarp();
             }
         } else {
-            {
+            if (BITMAP) {
+                // clear the words that cover [l_q, r_q]
+                const int w0 = l_q >> 5, w1 = r_q >> 5;
+                for (int i = w0 + lane; i <= w1; i += 32) bitmap[i] = 0u;
+            } else {
                 uint4* h4 = reinterpret_cast<uint4*>(S.hash);
                 const uint4 e4 = make_uint4(HASH_EMPTY, HASH_EMPTY, HASH_EMPTY, HASH_EMPTY);
                 for (int i = lane; i < (hash_slots >> 2); i += 32) h4[i] = e4;
@@ -150,7 +195,7 @@ frog_search_kernel(const FrogSearchArgs A) {
             {
                 const uint32_t ep = entry_point(A.seed, (uint32_t)l_q, (uint32_t)r_q, lane);
                 bool keep = lane < A.epn;
-                if (keep) keep = visited_insert(S.hash, A.hash_bits, ep, forgets);
+                if (keep) keep = visited_test_and_set<BITMAP>(S, bitmap, A.hash_bits, ep, forgets);
                 const uint32_t M = __ballot_sync(FULL, keep);
                 if (keep) S.cand[__popc(M & lt_mask)] = ep;
                 ns = __popc(M);
@@ -158,8 +203,7 @@ frog_search_kernel(const FrogSearchArgs A) {
             }
             FROG_PHASE(0);
             n_dist += ns;
-            int first = evaluate_and_merge<EPL>(A, S, ns, 0u, lane);
-            FROG_PHASE(3);
+            int first = EVAL(ns, 0u);
             // lines 7-17
             while (first < A.ef_s) {
                 if ((int)n_exp >= A.max_iters) { st |= FROG_ST_ITER_CAP; break; }
@@ -170,9 +214,11 @@ frog_search_kernel(const FrogSearchArgs A) {
                 // fetched per round trip); predicate "not empty and l_q <= v <= r_q" as one
                 // unsigned compare (the empty entry 0xFFFFFFFF minus l_q exceeds any span);
                 // ballot + popc give the admitted prefix under budget B.  Lines 12-13: each
-                // admitted lane applies the visited check where it stands; survivors are
-                // compacted into S.cand.
+                // admitted lane applies the visited check where it stands (it stays lazy: entries
+                // already evaluated still consume budget); survivors are compacted into S.cand.
                 const uint32_t* hot = A.enc + ((size_t)u * A.H + L_start) * A.m;
+                // a trace record is appended only while 66 words (header + 64 entries) remain
+                const bool rec_ok = (MODE == MODE_TRACE) && trace_ok && (trace_len + 66 <= (uint32_t)A.trace_cap - 1);
                 int cnt = 0, scanned = 0;
                 ns = 0;
                 for (int c0 = 0; c0 < total && cnt < A.B; c0 += 64) {
@@ -188,12 +234,11 @@ frog_search_kernel(const FrogSearchArgs A) {
                         const int a = min(__popc(M), A.B - cnt);
                         const bool admitted = pred && (__popc(M & lt_mask) < a);
                         if (MODE == MODE_TRACE) {
-                            if (trace_ok && admitted && 3 + trace_len + cnt + 16 < (uint32_t)A.trace_cap)
-                                trace_row[3 + trace_len + cnt + __popc(M & lt_mask)] = v;
+                            if (rec_ok && admitted) trace_row[3 + trace_len + cnt + __popc(M & lt_mask)] = v;
                         }
                         FROG_PHASE(1);
                         bool keep = admitted;
-                        if (keep) keep = visited_insert(S.hash, A.hash_bits, v, forgets);
+                        if (keep) keep = visited_test_and_set<BITMAP>(S, bitmap, A.hash_bits, v, forgets);
                         const uint32_t K = __ballot_sync(FULL, keep);
                         if (keep) S.cand[ns + __popc(K & lt_mask)] = v;
                         ns += __popc(K);
@@ -208,16 +253,14 @@ frog_search_kernel(const FrogSearchArgs A) {
                 n_en += cnt;
                 n_dist += ns;
                 if (MODE == MODE_TRACE) {
-                    // records are appended until the first one that does not fit
-                    if (trace_ok && trace_len + 2 + cnt <= (uint32_t)A.trace_cap - 1) {
+                    if (rec_ok) {
                         if (lane == 0) { trace_row[1 + trace_len] = u; trace_row[2 + trace_len] = (uint32_t)cnt; }
                         trace_len += 2 + cnt;
                     } else {
                         trace_ok = false;
                     }
                 }
-                first = evaluate_and_merge<EPL>(A, S, ns, 0u, lane);      // lines 14-17
-                FROG_PHASE(3);
+                first = EVAL(ns, 0u);   // lines 14-17
             }
         }
 
@@ -248,8 +291,8 @@ frog_search_kernel(const FrogSearchArgs A) {
             }
             if (MODE == MODE_TRACE) trace_row[0] = trace_len;
             if (MODE == MODE_PROFILE) {
-                trace_row[0] = 5;
-                for (int i = 0; i < 5; ++i) trace_row[1 + i] = (uint32_t)min(t_ph[i], 0xFFFFFFFFll);
+                trace_row[0] = 6;
+                for (int i = 0; i < 6; ++i) trace_row[1 + i] = (uint32_t)min(t_ph[i], 0xFFFFFFFFll);
             }
         }
         __syncwarp();
@@ -259,14 +302,14 @@ frog_search_kernel(const FrogSearchArgs A) {
 
 typedef void (*kernel_fn)(const FrogSearchArgs);
 
-template <int MODE>
+template <int MODE, bool BITMAP>
 kernel_fn pick_kernel(int ef_s, int* pool_slots) {
-    if (ef_s <= 32) { *pool_slots = 32; return frog_search_kernel<1, MODE>; }
-    if (ef_s <= 64) { *pool_slots = 64; return frog_search_kernel<2, MODE>; }
-    if (ef_s <= 128) { *pool_slots = 128; return frog_search_kernel<4, MODE>; }
-    if (ef_s <= 256) { *pool_slots = 256; return frog_search_kernel<8, MODE>; }
+    if (ef_s <= 32) { *pool_slots = 32; return frog_search_kernel<1, MODE, BITMAP>; }
+    if (ef_s <= 64) { *pool_slots = 64; return frog_search_kernel<2, MODE, BITMAP>; }
+    if (ef_s <= 128) { *pool_slots = 128; return frog_search_kernel<4, MODE, BITMAP>; }
+    if (ef_s <= 256) { *pool_slots = 256; return frog_search_kernel<8, MODE, BITMAP>; }
     *pool_slots = 512;
-    return frog_search_kernel<16, MODE>;
+    return frog_search_kernel<16, MODE, BITMAP>;
 }
 
 struct LaunchPlan {
@@ -275,12 +318,19 @@ struct LaunchPlan {
     size_t smem;
 };
 
-int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, int mode, int nq, LaunchPlan* out) {
+int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, int mode, bool bitmap, int nq,
+                LaunchPlan* out) {
     int pool_slots = 0;
-    kernel_fn fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE>(beam_width, &pool_slots)
-                 : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE>(beam_width, &pool_slots)
-                                        : pick_kernel<MODE_FAST>(beam_width, &pool_slots);
-    size_t smem = warp_smem_bytes(pool_slots, ix->info.d_pad, P.hash_bits) * WARPS_PER_CTA;
+    kernel_fn fn;
+    if (bitmap)
+        fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, true>(beam_width, &pool_slots)
+           : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, true>(beam_width, &pool_slots)
+                                  : pick_kernel<MODE_FAST, true>(beam_width, &pool_slots);
+    else
+        fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, false>(beam_width, &pool_slots)
+           : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, false>(beam_width, &pool_slots)
+                                  : pick_kernel<MODE_FAST, false>(beam_width, &pool_slots);
+    size_t smem = warp_smem_bytes(pool_slots, ix->info.d_pad, P.hash_bits, bitmap) * WARPS_PER_CTA;
     if (smem > 227 * 1024) return FROG_ERR_UNSUPPORTED;
     FROG_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
@@ -297,6 +347,12 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
     out->ctas_per_sm = per_sm;
     out->smem = smem;
     return FROG_OK;
+}
+
+// per-warp visited slab: one bit per rank, padded to 128 bytes
+size_t bitmap_words_per_slot(const frog_index* ix) {
+    size_t words = ((size_t)ix->info.n + 31) / 32;
+    return (words + 31) & ~(size_t)31;
 }
 
 }  // namespace
@@ -320,8 +376,30 @@ int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in
         P.hash_bits = bits;
     }
     if (P.hash_bits < 6 || P.hash_bits > 15) return FROG_ERR_INVALID_ARG;
+    if (P.visited != FROG_VISITED_AUTO && P.visited != FROG_VISITED_BITMAP && P.visited != FROG_VISITED_HASH)
+        return FROG_ERR_INVALID_ARG;
     (void)ix;
     *out = P;
+    return FROG_OK;
+}
+
+// Make sure the index owns a visited slab for `slots` resident warps.  Grows (cudaFree + cudaMalloc,
+// after synchronising the device) only when a launch needs more slots than any launch before it.
+int ensure_bitmap(const frog_index* cix, size_t slots) {
+    frog_index* ix = const_cast<frog_index*>(cix);
+    const size_t words = bitmap_words_per_slot(ix);
+    if (ix->d_bitmap && ix->bitmap_slots >= slots) return FROG_OK;
+    FROG_CUDA_TRY(cudaDeviceSynchronize());
+    if (ix->d_bitmap) FROG_CUDA_TRY(cudaFree(ix->d_bitmap));
+    ix->d_bitmap = nullptr;
+    ix->bitmap_slots = 0;
+    cudaError_t e = cudaMalloc(&ix->d_bitmap, slots * words * sizeof(uint32_t));
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        set_cuda_error(e);
+        return FROG_ERR_NOMEM;
+    }
+    ix->bitmap_slots = slots;
     return FROG_OK;
 }
 
@@ -335,7 +413,7 @@ extern "C" int frog_search_launch_info(const frog_index_t* index, int beam_width
     if (rc) return rc;
     FROG_CUDA_TRY(cudaSetDevice(index->info.device));
     LaunchPlan plan;
-    rc = plan_launch(index, beam_width, P, MODE_FAST, 0, &plan);
+    rc = plan_launch(index, beam_width, P, MODE_FAST, P.visited != FROG_VISITED_HASH, 0, &plan);
     if (rc) return rc;
     if (grid) *grid = plan.grid;
     if (block) *block = plan.block;
@@ -357,10 +435,20 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     int rc = froghost::resolve_params(index, beam_width, params, &P);
     if (rc) return rc;
     FROG_CUDA_TRY(cudaSetDevice(index->info.device));
+    const int mode = !trace ? MODE_FAST : (P.debug_flags & 1) ? MODE_PROFILE : MODE_TRACE;
+    bool bitmap = P.visited != FROG_VISITED_HASH;
     LaunchPlan plan;
-    const int mode = !trace ? MODE_FAST : (P.reserved & 1) ? MODE_PROFILE : MODE_TRACE;
-    rc = plan_launch(index, beam_width, P, mode, nq, &plan);
+    rc = plan_launch(index, beam_width, P, mode, bitmap, nq, &plan);
     if (rc) return rc;
+    if (bitmap) {
+        rc = froghost::ensure_bitmap(index, (size_t)plan.grid * WARPS_PER_CTA);
+        if (rc == FROG_ERR_NOMEM && P.visited == FROG_VISITED_AUTO) {
+            // no room for the slabs: fall back to the shared-memory table
+            bitmap = false;
+            rc = plan_launch(index, beam_width, P, mode, false, nq, &plan);
+        }
+        if (rc) return rc;
+    }
 
     FrogSearchArgs A;
     A.sorted_attr = index->d_sorted_attr;
@@ -391,6 +479,8 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     A.trace = trace;
     A.trace_cap = trace_cap;
     A.work_counter = index->d_work;
+    A.bitmap = bitmap ? index->d_bitmap : nullptr;
+    A.bitmap_words = bitmap_words_per_slot(index);
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     FROG_CUDA_TRY(cudaMemsetAsync(index->d_work, 0, sizeof(unsigned int), s));
