@@ -35,7 +35,8 @@ enum {
     FROG_ERR_FORMAT = 3,        /* magic, version, sizes or offsets inconsistent */
     FROG_ERR_NOMEM = 4,         /* host or device allocation failed */
     FROG_ERR_CUDA = 5,          /* a CUDA runtime call failed; see frog_last_cuda_error() */
-    FROG_ERR_UNSUPPORTED = 6    /* parameter combination the kernels do not cover */
+    FROG_ERR_UNSUPPORTED = 6,   /* parameter combination the kernels do not cover */
+    FROG_ERR_TOO_LARGE = 7      /* frog_search_static: the index exceeds FROG_STATIC_MAX_N objects */
 };
 
 /* Limits of the search kernels. */
@@ -149,6 +150,36 @@ int frog_exact_search(const frog_index_t* index, const float* queries, const int
 int frog_search_host(frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
                      int nq, int k, int beam_width, const frog_params_t* params /* HOST, may be null */,
                      int32_t* out_ids, float* out_dists, void* stream);
+
+/* frog_search_static: frog_search_ex (without the optional per-query outputs) for callers that
+ * cannot allocate device memory at search time.  The paper has no counterpart; this entry point
+ * exists for deployment reasons only.  Who needs it: a serving loop or a captured stream where the
+ * device-wide synchronisation hidden in cudaMalloc/cudaFree is not acceptable; a plug-in that was
+ * handed a fixed memory budget by its host application; a process that shares the GPU with
+ * another framework's caching allocator, which has already claimed the free memory, so that an
+ * allocation here would fail or fragment it.
+ *
+ * All scratch of the search (the work counter and the per-warp visited bitmaps) lives in one
+ * file-scope device array inside the library, 16 MiB + 256 bytes, which every GPU that loads the
+ * library holds until the process exits.  The call itself performs no cudaMalloc, cudaFree or
+ * other allocating routine.  Consequences:
+ *   - an index may hold at most FROG_STATIC_MAX_N objects, so that the bitmaps of at least
+ *     FROG_STATIC_MIN_SLOTS warps fit; larger indexes are refused with FROG_ERR_TOO_LARGE.  The
+ *     number of resident warps is capped by what fits, so large indexes run with less
+ *     parallelism than frog_search gives them;
+ *   - the first call on a device looks up the device address of the array (once per device,
+ *     with that device current); make that first call before starting any stream capture;
+ *   - every call, on every index and stream of the device, shares the one array, and the array
+ *     keeps what the last call left in it.  The call resets the counter and each warp clears the
+ *     bitmap words it is about to use, so consecutive calls are independent; calls that overlap
+ *     on the GPU race on it and must be serialised by the caller.
+ * Arguments, results and errors otherwise as frog_search_ex; `params` may be null;
+ * params->visited is ignored (the bitmap form is always used). */
+#define FROG_STATIC_MAX_N 2097152 /* objects: 256 KiB of visited bits per warp */
+#define FROG_STATIC_MIN_SLOTS 64  /* resident warps guaranteed at FROG_STATIC_MAX_N */
+int frog_search_static(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
+                       int nq, int k, int beam_width, const frog_params_t* params,
+                       int32_t* out_ids, float* out_dists, void* stream);
 
 /* Launch shape of the search kernel for the given beam width (for reporting): CTAs, threads per
  * CTA, dynamic shared memory per CTA, query slots resident per SM. */

@@ -188,6 +188,27 @@ class Index:
             raise FrogError(rc, "frog_search")
         return out_ids, out_dists
 
+    def search_static(self, queries, lo, hi, k: int, beam_width: int, out_ids=None, out_dists=None,
+                      stream=None, params: Optional[Params] = None):
+        """The search through ``frog_search_static``: same results as :meth:`search`, but all scratch
+        sits in a fixed 16 MiB device array inside the library, so the call never allocates device
+        memory (for callers under stream capture, with a fixed memory budget, or next to another
+        allocator that owns the free memory).  Output tensors are still the caller's: pass
+        ``out_ids``/``out_dists`` to keep this wrapper allocation-free too.  Indexes of more than
+        2,097,152 objects are refused; overlapping calls on one device must be serialised."""
+        import torch
+        nq = self._check(queries, lo, hi)
+        if out_ids is None:
+            out_ids = torch.empty((nq, k), dtype=torch.int32, device=queries.device)
+        if out_dists is None:
+            out_dists = torch.empty((nq, k), dtype=torch.float32, device=queries.device)
+        rc = _lib.frog_search_static(self._h, _ptr(queries), _ptr(lo), _ptr(hi), C.c_int(nq), C.c_int(k),
+                                     C.c_int(beam_width), C.byref(params) if params is not None else None,
+                                     _ptr(out_ids), _ptr(out_dists), _stream_ptr(stream))
+        if rc:
+            raise FrogError(rc, "frog_search_static")
+        return out_ids, out_dists
+
     def exact_search(self, queries, lo, hi, k: int, out_ids=None, out_dists=None, stream=None):
         """Exact filtered kNN by slab scan (ground truth / pre-filtering reference)."""
         import torch

@@ -97,6 +97,7 @@ extern "C" const char* frog_strerror(int code) {
         case FROG_ERR_NOMEM: return "out of memory";
         case FROG_ERR_CUDA: return "CUDA error";
         case FROG_ERR_UNSUPPORTED: return "unsupported parameters";
+        case FROG_ERR_TOO_LARGE: return "index too large for the static scratch (more than 2097152 objects)";
         default: return "unknown error";
     }
 }

@@ -15,6 +15,7 @@
 //     crowded table forgets entries, which costs repeated distance evaluations, never results).
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "frog_device.cuh"
 #include "frog_internal.h"
@@ -493,4 +494,112 @@ extern "C" int frog_search(const frog_index_t* index, const float* queries, cons
                            int nq, int k, int beam_width, int32_t* out_ids, float* out_dists, void* stream) {
     return frog_search_ex(index, queries, lo, hi, nq, k, beam_width, nullptr, out_ids, out_dists,
                           nullptr, nullptr, nullptr, 0, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// frog_search_static: the same search with every byte of scratch in a fixed device array.
+//
+// Some callers must not allocate device memory while they search: code running under a stream
+// capture or inside a latency-critical serving loop where cudaMalloc's implicit synchronisation
+// is not acceptable, plug-ins whose host hands them a fixed memory budget, and processes that
+// run next to another framework's caching allocator which already owns the free memory.  For them
+// the work counter and the per-warp visited slabs live in the array below.  Its size is fixed at
+// compile time (16 MiB + 256 B, held by every GPU that loads this library until the process
+// exits), so the call limits the number of resident warps to the slabs that fit and refuses
+// indexes whose slab is too large for at least FROG_STATIC_MIN_SLOTS warps.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t STATIC_HEADER_WORDS = 64;                          // work counter + spare
+constexpr size_t STATIC_SLAB_WORDS = (size_t)4 << 20;               // 4 Mi words = 16 MiB of visited bits
+static __device__ __align__(256) uint32_t g_static_scratch[STATIC_HEADER_WORDS + STATIC_SLAB_WORDS];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+uint32_t* g_static_ptr[STATIC_MAX_DEVICES] = {};                    // device address of the array, per device
+std::mutex g_static_mutex;
+
+// The array's name is only a host-side handle in host code; the device address must be asked
+// for, once per device, with that device current.
+int static_scratch_for_device(int device, uint32_t** out) {
+    if (device < 0 || device >= STATIC_MAX_DEVICES) return FROG_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) {
+            froghost::set_cuda_error(e);
+            return FROG_ERR_CUDA;
+        }
+        g_static_ptr[device] = static_cast<uint32_t*>(p);
+    }
+    *out = g_static_ptr[device];
+    return FROG_OK;
+}
+
+}  // namespace
+
+extern "C" int frog_search_static(const frog_index_t* index, const float* queries, const int32_t* lo,
+                                  const int32_t* hi, int nq, int k, int beam_width, const frog_params_t* params,
+                                  int32_t* out_ids, float* out_dists, void* stream) {
+    if (!index || nq < 0) return FROG_ERR_INVALID_ARG;
+    if (k < 1 || beam_width < 1 || beam_width > FROG_MAX_BEAM_WIDTH || k > beam_width) return FROG_ERR_INVALID_ARG;
+    if (nq == 0) return FROG_OK;
+    if (!queries || !lo || !hi || !out_ids || !out_dists) return FROG_ERR_INVALID_ARG;
+    frog_params_t P;
+    int rc = froghost::resolve_params(index, beam_width, params, &P);
+    if (rc) return rc;
+    // the slab of one warp must fit FROG_STATIC_MIN_SLOTS times: n <= FROG_STATIC_MAX_N
+    if (index->info.n > FROG_STATIC_MAX_N) return FROG_ERR_TOO_LARGE;
+    const size_t words = bitmap_words_per_slot(index);
+    const size_t fit = STATIC_SLAB_WORDS / words;
+    if (fit < FROG_STATIC_MIN_SLOTS) return FROG_ERR_TOO_LARGE;
+    FROG_CUDA_TRY(cudaSetDevice(index->info.device));
+    uint32_t* scratch = nullptr;
+    rc = static_scratch_for_device(index->info.device, &scratch);
+    if (rc) return rc;
+    LaunchPlan plan;
+    rc = plan_launch(index, beam_width, P, MODE_FAST, true, nq, &plan);
+    if (rc) return rc;
+    const int max_ctas = (int)(fit / WARPS_PER_CTA);
+    if (plan.grid > max_ctas) plan.grid = max_ctas;
+
+    FrogSearchArgs A;
+    A.sorted_attr = index->d_sorted_attr;
+    A.rank2id = index->d_rank2id;
+    A.vectors = index->d_vectors;
+    A.enc = index->d_enc;
+    A.n = (int)index->info.n;
+    A.d = index->info.d;
+    A.d_pad = index->info.d_pad;
+    A.H = index->info.H;
+    A.m = index->info.m;
+    A.queries = queries;
+    A.lo = lo;
+    A.hi = hi;
+    A.nq = nq;
+    A.k = k;
+    A.ef_s = beam_width;
+    A.epn = P.epn;
+    A.B = P.budget;
+    A.max_iters = P.max_iters;
+    A.no_hotspot = P.no_hotspot;
+    A.hash_bits = P.hash_bits;
+    A.seed = P.seed;
+    A.out_ids = out_ids;
+    A.out_dists = out_dists;
+    A.status = nullptr;
+    A.stats = nullptr;
+    A.trace = nullptr;
+    A.trace_cap = 0;
+    A.work_counter = scratch;                               // word 0 of the header
+    A.bitmap = scratch + STATIC_HEADER_WORDS;
+    A.bitmap_words = words;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the array keeps what the previous call left: the counter must restart at zero; every warp
+    // clears the slab words of a query's range itself before using them
+    FROG_CUDA_TRY(cudaMemsetAsync(scratch, 0, sizeof(unsigned int), s));
+    plan.fn<<<plan.grid, plan.block, plan.smem, s>>>(A);
+    FROG_CUDA_TRY(cudaGetLastError());
+    return FROG_OK;
 }
