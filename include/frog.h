@@ -84,6 +84,8 @@ typedef struct {
 #define FROG_ST_EXACT 2u     /* range holds <= beam_width objects: answered by exact scan */
 #define FROG_ST_ITER_CAP 4u  /* expansion cap hit; the current pool was returned */
 #define FROG_ST_SHORT 8u     /* fewer than k results; tail is padding */
+#define FROG_ST_COPY_TIMEOUT 32u /* a bulk copy into shared memory did not complete within the kernel's
+                                    polling limit; the row's results are not valid (never expected) */
 #define FROG_ST_FORGOT 16u   /* the visited table overflowed and dropped entries: some distances were
                                 evaluated twice; the results are unaffected */
 

@@ -5,10 +5,12 @@
 //   hotspot_layers     Alg. 3 HotspotLocalization with Eq. 6 evaluated in integers
 //   visited_insert     the hash check of Alg. 2 line 12
 //   batch_dist2        gather of <= 16 rows with 16-byte loads + fp32 squared L2, 8-lane teams
+//   staged_dist2       the same distances with the rows staged in shared memory by TMA bulk copies
 //   merge_batch        sort `new`, MergeTopEfS and "first unexpanded" of Alg. 2 lines 15-17
 #pragma once
 
 #include <cstdint>
+#include <cstdio>
 #include <cuda_runtime.h>
 
 namespace frogdev {
@@ -195,6 +197,119 @@ __device__ __forceinline__ float batch_dist2(const float* __restrict__ vectors, 
             accB = accB + __shfl_xor_sync(FULL, accB, 1);
             const float vb = __shfl_sync(FULL, accB, src);
             if ((lane >> 2) == r0 + 1) out = vb;
+        }
+    }
+    return out;
+}
+
+// ---- TMA bulk copies (global -> shared) completing on an mbarrier ----------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// One thread asks the copy engine for `bytes` (multiple of 16, both addresses 16-byte aligned);
+// the bytes are credited to the mbarrier when they have landed in shared memory.
+__device__ __forceinline__ void tma_load_1d(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// Wait for the phase of parity `phase`; bounded: gives up after ~2^22 polls and reports false
+// (the caller flags the query instead of hanging the GPU).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t phase) {
+    const uint32_t addr = smem_u32(bar);
+    for (int it = 0; it < (1 << 22); ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(addr), "r"(phase) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// Squared L2 distances of up to 32 rows, rows staged in shared memory by the copy engine.
+// Lane j < ns holds the rank of row j in `my_rank`; on return lane j holds its distance.
+// The ranks of one call must be pairwise distinct (see evaluate_and_merge).
+// Rows are taken STAGE_ROWS at a time and, for long rows, in column chunks of at most
+// STAGE_CHUNK bytes: one elected lane per row issues a bulk copy of the chunk into the stage
+// buffer, all copies of a pass complete on one mbarrier, then every 8-lane team reduces its rows
+// from shared memory.  The arithmetic order is the one of batch_dist2 (lane s of a team takes the
+// 4-float groups g = s, s+8, ... in increasing g, fused multiply-adds, butterfly 4-2-1), so both
+// routines return identical bits.  `phase` is the running parity of the warp's mbarrier.
+constexpr int STAGE_CHUNK = 512;     // bytes of one row in flight per pass
+template <int STAGE_ROWS>
+__device__ __forceinline__ float staged_dist2(const float* __restrict__ vectors, int d_pad, const float4* qs,
+                                              float4* stage, uint64_t* bar, uint32_t& phase, bool& ok,
+                                              uint32_t my_rank, int ns, int lane) {
+    static_assert(STAGE_ROWS == 8 || STAGE_ROWS == 16, "rows per pass");
+    const int team = lane >> 3, sub = lane & 7;
+    const int row_bytes = d_pad * 4;
+    float out = 0.f;
+#pragma unroll 1
+    for (int r0 = 0; r0 < ns; r0 += STAGE_ROWS) {
+        const int nrows = min(STAGE_ROWS, ns - r0);
+        // rank of the row this lane would copy (lane r copies row r0 + r)
+        const uint32_t copy_rank = __shfl_sync(FULL, my_rank, (r0 + lane) & 31);
+        const char* src_row = reinterpret_cast<const char*>(vectors) + (size_t)copy_rank * (size_t)row_bytes;
+        float acc[STAGE_ROWS / 4];
+#pragma unroll
+        for (int i = 0; i < STAGE_ROWS / 4; ++i) acc[i] = 0.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < row_bytes; c0 += STAGE_CHUNK) {
+            const int cbytes = min(STAGE_CHUNK, row_bytes - c0);
+            __syncwarp();                                   // every lane is done reading the stage buffer
+            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(nrows * cbytes));
+            __syncwarp();
+            if (lane < nrows)
+                tma_load_1d(reinterpret_cast<char*>(stage) + lane * STAGE_CHUNK, src_row + c0, (uint32_t)cbytes, bar);
+            {
+                const bool done_ = mbar_wait(bar, phase);
+#ifdef FROG_DEBUG_TMA
+                if (!done_) printf("timeout blk %d thr %d lane %d phase %u ns %d r0 %d nrows %d c0 %d cbytes %d rank %u\n",
+                                   blockIdx.x, threadIdx.x, lane, phase, ns, r0, nrows, c0, cbytes, copy_rank);
+#endif
+                ok = done_ && ok;
+            }
+            phase ^= 1u;
+            const int g_lo = c0 >> 4, g_n = cbytes >> 4;    // 4-float groups of this chunk
+#pragma unroll
+            for (int i = 0; i < STAGE_ROWS / 4; ++i) {
+                const int r = i * 4 + team;
+                if (r < nrows) {
+                    const float4* xrow = stage + r * (STAGE_CHUNK / 16);
+#pragma unroll 4
+                    for (int g = sub; g < g_n; g += 8) {
+                        const float4 x = xrow[g];
+                        const float4 q = qs[g_lo + g];
+                        float t;
+                        t = x.x - q.x; acc[i] = fmaf(t, t, acc[i]);
+                        t = x.y - q.y; acc[i] = fmaf(t, t, acc[i]);
+                        t = x.z - q.z; acc[i] = fmaf(t, t, acc[i]);
+                        t = x.w - q.w; acc[i] = fmaf(t, t, acc[i]);
+                    }
+                }
+            }
+        }
+        // row r0 + j was reduced by team j & 3 as its (j >> 2)-th row
+        const int src = (lane & 3) << 3;
+#pragma unroll
+        for (int i = 0; i < STAGE_ROWS / 4; ++i) {
+            if (i * 4 < nrows) {
+                float a = acc[i];
+                a = a + __shfl_xor_sync(FULL, a, 4);
+                a = a + __shfl_xor_sync(FULL, a, 2);
+                a = a + __shfl_xor_sync(FULL, a, 1);
+                // the result for row r0 + i*4 + t sits in team t; hand it to lane r0 + i*4 + t
+                const float v = __shfl_sync(FULL, a, src);
+                if (lane >= r0 && ((lane - r0) >> 2) == i && lane - r0 < nrows) out = v;
+            }
         }
     }
     return out;

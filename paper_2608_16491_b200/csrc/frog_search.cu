@@ -37,15 +37,24 @@ constexpr int WARPS_PER_CTA = 2;
 #endif
 constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2;
 
+#ifndef FROG_STAGE_ROWS
+#define FROG_STAGE_ROWS 8     // rows the copy engine stages per pass (8 or 16), 512 bytes each
+#endif
+constexpr int STAGE_BYTES = FROG_STAGE_ROWS * STAGE_CHUNK;
+
+// per-warp shared memory: pool | candidate list | mbarrier, its phase, a failure flag | query | stage | hash
 struct WarpSmem {
     uint64_t* pool;
     uint32_t* cand;
+    uint64_t* bar;       // bar[0] = mbarrier; the two words after it: phase parity, copy-timeout flag
     float4* q;
+    float4* stage;
     uint32_t* hash;
 };
 
 inline size_t warp_smem_bytes(int pool_slots, int d_pad, int hash_bits, bool bitmap) {
-    return (size_t)pool_slots * 8 + 32 * 4 + (size_t)d_pad * 4 + (bitmap ? 0 : ((size_t)4 << hash_bits));
+    return (size_t)pool_slots * 8 + 32 * 4 + 16 + (size_t)d_pad * 4 + STAGE_BYTES +
+           (bitmap ? 0 : ((size_t)4 << hash_bits));
 }
 
 // entry point j of a query range: stateless mixer of (seed, l_q, r_q, j), top 32 bits scaled
@@ -78,18 +87,37 @@ __device__ __forceinline__ bool visited_test_and_set(const WarpSmem& S, uint32_t
 // three places of the kernel and inlining every copy costs registers and instruction cache.
 template <int EPL>
 __device__ FROG_EVAL_INLINE int evaluate_and_merge(const float* __restrict__ vectors, int d_pad, int ef_s,
-                                                   uint64_t* pool, const uint32_t* cand, const float4* qs,
-                                                   int ns, uint32_t new_flag, long long* t_dist) {
+                                                   uint64_t* pool, const uint32_t* cand, uint64_t* bar,
+                                                   const float4* qs, float4* stage,
+                                                   int ns, uint32_t new_flag, bool dedupe, long long* t_dist) {
     const int lane = lane_id();
-    const uint32_t id = (lane < ns) ? cand[lane] : 0u;
+    uint32_t id = (lane < ns) ? cand[lane] : 0u;
+    if (dedupe) {
+        // The shared-memory visited table can let the same rank through twice in one batch once it
+        // starts dropping entries.  Two bulk copies of one source row completing on the same
+        // mbarrier were observed to leave the barrier incomplete (the wait ran into its polling
+        // limit), so repeated ranks are squeezed out before the gather.  The bitmap form never
+        // produces repeats.
+        const uint32_t same = __match_any_sync(FULL, (lane < ns) ? id : (0x80000000u | (uint32_t)lane));
+        const bool first_copy = (lane < ns) && ((__ffs(same) - 1) == lane);
+        const uint32_t keep_mask = __ballot_sync(FULL, first_copy);
+        const int src_lane = __fns(keep_mask, 0, lane + 1);          // lane holding the (lane+1)-th kept rank
+        const uint32_t moved = __shfl_sync(FULL, id, src_lane & 31);
+        ns = __popc(keep_mask);
+        id = (lane < ns) ? moved : 0u;
+    }
     float d2 = 0.f;
-    if (ns > 0) d2 = batch_dist2<FROG_NG>(vectors, d_pad, qs, id, min(ns, 16), lane);
-    if (ns > 16) {
-        // rows 16..31: computed with the ids moved down to lanes 0..15, result moved back up
-        const uint32_t id_hi = __shfl_down_sync(FULL, id, 16);
-        const float d_hi = batch_dist2<FROG_NG>(vectors, d_pad, qs, id_hi, ns - 16, lane);
-        const float up = __shfl_up_sync(FULL, d_hi, 16);
-        if (lane >= 16) d2 = up;
+    if (ns > 0) {
+        uint32_t* bar_words = reinterpret_cast<uint32_t*>(bar + 1);
+        __syncwarp();                       // lane 0's update of the parity in the previous call
+        uint32_t phase = bar_words[0];
+        bool ok = true;
+        d2 = staged_dist2<FROG_STAGE_ROWS>(vectors, d_pad, qs, stage, bar, phase, ok, id, ns, lane);
+        __syncwarp();                       // every lane has read the old parity
+        if (lane == 0) {
+            bar_words[0] = phase;
+            if (!ok) bar_words[1] = 1u;
+        }
     }
     const uint64_t key = (lane < ns) ? make_key(d2, id, new_flag) : KEY_EMPTY;
     if (t_dist) *t_dist = clock64();
@@ -104,13 +132,21 @@ frog_search_kernel(const FrogSearchArgs A) {
     const int warp = threadIdx.x >> 5;
     constexpr int POOL = 32 * EPL;
     const int hash_slots = BITMAP ? 0 : (1 << A.hash_bits);
-    const size_t per_warp = (size_t)POOL * 8 + 32 * 4 + (size_t)A.d_pad * 4 + (size_t)hash_slots * 4;
+    const size_t per_warp = (size_t)POOL * 8 + 32 * 4 + 16 + (size_t)A.d_pad * 4 + STAGE_BYTES + (size_t)hash_slots * 4;
     unsigned char* base = smem_raw + per_warp * warp;
     WarpSmem S;
     S.pool = reinterpret_cast<uint64_t*>(base);
     S.cand = reinterpret_cast<uint32_t*>(S.pool + POOL);
-    S.q = reinterpret_cast<float4*>(S.cand + 32);
-    S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<float*>(S.q) + A.d_pad);
+    S.bar = reinterpret_cast<uint64_t*>(S.cand + 32);
+    S.q = reinterpret_cast<float4*>(S.bar + 2);
+    S.stage = reinterpret_cast<float4*>(reinterpret_cast<float*>(S.q) + A.d_pad);
+    S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(S.stage) + STAGE_BYTES);
+    if (lane == 0) {
+        mbar_init(S.bar, 1u);
+        reinterpret_cast<uint32_t*>(S.bar + 1)[0] = 0u;   // phase parity
+        reinterpret_cast<uint32_t*>(S.bar + 1)[1] = 0u;   // copy-timeout flag
+    }
+    __syncwarp();
     uint32_t* bitmap = BITMAP ? A.bitmap + (size_t)(blockIdx.x * WARPS_PER_CTA + warp) * A.bitmap_words : nullptr;
     const uint32_t lt_mask = (1u << lane) - 1u;
 
@@ -134,8 +170,8 @@ frog_search_kernel(const FrogSearchArgs A) {
         // distance + merge call; in profile builds the time is split at the end of the distances
         long long t_split = 0;
         auto EVAL = [&](int ns_, uint32_t flag_) {
-            int f_ = evaluate_and_merge<EPL>(A.vectors, A.d_pad, A.ef_s, S.pool, S.cand, S.q, ns_, flag_,
-                                             MODE == MODE_PROFILE ? &t_split : nullptr);
+            int f_ = evaluate_and_merge<EPL>(A.vectors, A.d_pad, A.ef_s, S.pool, S.cand, S.bar, S.q, S.stage, ns_,
+                                             flag_, !BITMAP, MODE == MODE_PROFILE ? &t_split : nullptr);
             if (MODE == MODE_PROFILE) {
                 long long n_ = clock64();
                 t_ph[3] += t_split - t_mark;
@@ -283,6 +319,7 @@ frog_search_kernel(const FrogSearchArgs A) {
         got = __reduce_add_sync(FULL, got);
         if (got < A.k) st |= FROG_ST_SHORT;
         if (__any_sync(FULL, forgets != 0)) st |= FROG_ST_FORGOT;   // counted per lane
+        if (reinterpret_cast<uint32_t*>(S.bar + 1)[1]) st |= FROG_ST_COPY_TIMEOUT;
         FROG_PHASE(4);
         if (lane == 0) {
             if (A.status) A.status[q] = st;
