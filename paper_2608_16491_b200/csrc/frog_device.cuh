@@ -315,16 +315,30 @@ __device__ __forceinline__ float staged_dist2(const float* __restrict__ vectors,
     return out;
 }
 
+// two smallest values seen by a lane
+__device__ __forceinline__ void track2(int& m1, int& m2, int p) {
+    if (p < m1) { m2 = m1; m1 = p; }
+    else if (p < m2) m2 = p;
+}
+// warp-wide smallest and second smallest of the per-lane pairs (m1 <= m2), packed as
+// first | second << 16 (0xFFFF = none)
+__device__ __forceinline__ uint32_t first_two(int m1, int m2) {
+    const unsigned a = min((unsigned)m1, 0xFFFFu), b = min((unsigned)m2, 0xFFFFu);
+    const unsigned f = __reduce_min_sync(FULL, a);
+    const unsigned s2 = __reduce_min_sync(FULL, a == f ? b : a);
+    return f | (s2 << 16);
+}
+
 // Alg. 2 lines 15-17 in one pass.  `pool` holds ef_s (<= 32*EPL) keys ascending by key | 1,
 // KEY_EMPTY at the tail; each lane brings at most one new key (KEY_EMPTY = none).  The final
 // position of a new key is (#pool keys below it) + (#new keys below it); of a pool key, its
 // index + (#new keys below it); everything landing at >= ef_s is dropped.  All counts come from
 // register compares and ballots: the new keys are broadcast one by one with shuffles, the lanes
 // hold the pool keys (lane l owns positions l, l+32, ...).  A new key equal to a pool key (a vertex
-// the visited table forgot) or to an earlier new key is discarded.  Returns the first position
-// whose flag is 0, NO_POS if none.
+// the visited table forgot) or to an earlier new key is discarded.  Returns the positions of the
+// first and of the second entry whose flag is 0, packed as first | second << 16 (0xFFFF = none).
 template <int EPL>
-__device__ __forceinline__ int merge_batch(uint64_t* pool, uint64_t my_key, int ef_s, int lane) {
+__device__ __forceinline__ uint32_t merge_batch(uint64_t* pool, uint64_t my_key, int ef_s, int lane) {
     uint64_t pk[EPL];
 #pragma unroll
     for (int e = 0; e < EPL; ++e) pk[e] = pool[lane + 32 * e];
@@ -332,12 +346,12 @@ __device__ __forceinline__ int merge_batch(uint64_t* pool, uint64_t my_key, int 
     const uint64_t worst = pool[ef_s - 1];
     if ((my_key | 1ull) >= (worst | 1ull)) my_key = KEY_EMPTY;
     uint32_t have = __ballot_sync(FULL, my_key != KEY_EMPTY);
-    int first = NO_POS;
+    int m1 = NO_POS, m2 = NO_POS;
     if (have == 0) {
 #pragma unroll
         for (int e = 0; e < EPL; ++e)
-            if (pk[e] != KEY_EMPTY && !(pk[e] & 1ull)) first = min(first, lane + 32 * e);
-        return (int)__reduce_min_sync(FULL, (unsigned)first);
+            if (pk[e] != KEY_EMPTY && !(pk[e] & 1ull)) track2(m1, m2, lane + 32 * e);
+        return first_two(m1, m2);
     }
     int add[EPL];
 #pragma unroll
@@ -377,7 +391,7 @@ __device__ __forceinline__ int merge_batch(uint64_t* pool, uint64_t my_key, int 
             const int p = lane + 32 * e + add[e];
             if (p < ef_s) {
                 if (add[e]) pool[p] = pk[e];
-                if (!(pk[e] & 1ull)) first = min(first, p);
+                if (!(pk[e] & 1ull)) track2(m1, m2, p);
             }
         }
     }
@@ -385,11 +399,26 @@ __device__ __forceinline__ int merge_batch(uint64_t* pool, uint64_t my_key, int 
         const int p = (32 * EPL - above) + rnew;
         if (p < ef_s) {
             pool[p] = my_key;
-            if (!(my_key & 1ull)) first = min(first, p);
+            if (!(my_key & 1ull)) track2(m1, m2, p);
         }
     }
     __syncwarp();
-    return (int)__reduce_min_sync(FULL, (unsigned)first);
+    return first_two(m1, m2);
+}
+
+// smallest key of the warp under the order key | 1 (KEY_EMPTY if no lane has one)
+__device__ __forceinline__ uint64_t warp_min_key(uint64_t key) {
+    const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key | 1u;
+    const uint32_t mhi = __reduce_min_sync(FULL, hi);
+    const uint32_t mlo = __reduce_min_sync(FULL, hi == mhi ? lo : 0xFFFFFFFFu);
+    return ((uint64_t)mhi << 32) | mlo;
+}
+
+__device__ __forceinline__ void prefetch_l1(const void* p) {
+    asm volatile("prefetch.global.L1 [%0];" ::"l"(p));
+}
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
 
 }  // namespace frogdev

@@ -37,6 +37,15 @@ constexpr int WARPS_PER_CTA = 2;
 #endif
 constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2;
 
+#ifndef FROG_ENC_PREFETCH
+#define FROG_ENC_PREFETCH 1   // 0: off, 1: prefetch the predicted vertex's ENC lines
+#endif
+#ifndef FROG_PREFETCH_FN
+#define FROG_PREFETCH_FN prefetch_l2
+#endif
+#ifndef FROG_ENC_LD
+#define FROG_ENC_LD ldg_stream_u32
+#endif
 #ifndef FROG_STAGE_ROWS
 #define FROG_STAGE_ROWS 8     // rows the copy engine stages per pass (8 or 16), 512 bytes each
 #endif
@@ -89,7 +98,9 @@ template <int EPL>
 __device__ FROG_EVAL_INLINE int evaluate_and_merge(const float* __restrict__ vectors, int d_pad, int ef_s,
                                                    uint64_t* pool, const uint32_t* cand, uint64_t* bar,
                                                    const float4* qs, float4* stage,
-                                                   int ns, uint32_t new_flag, bool dedupe, long long* t_dist) {
+                                                   int ns, uint32_t new_flag, bool dedupe,
+                                                   const uint32_t* enc_hot, size_t enc_stride, int enc_bytes,
+                                                   int next_pos, long long* t_dist) {
     const int lane = lane_id();
     uint32_t id = (lane < ns) ? cand[lane] : 0u;
     if (dedupe) {
@@ -121,7 +132,24 @@ __device__ FROG_EVAL_INLINE int evaluate_and_merge(const float* __restrict__ vec
     }
     const uint64_t key = (lane < ns) ? make_key(d2, id, new_flag) : KEY_EMPTY;
     if (t_dist) *t_dist = clock64();
-    return merge_batch<EPL>(pool, key, ef_s, lane);
+#if FROG_ENC_PREFETCH
+    if (enc_hot) {
+        // The vertex expanded next is the smaller of the best new key that enters the pool and the
+        // pool's next unexpanded entry: start fetching the first lines of its ENC rows now, so the
+        // fetch overlaps the merge.  A wrong guess only wastes the prefetch.
+        uint64_t guess = warp_min_key(key);
+        const uint64_t worst = pool[ef_s - 1];
+        if ((guess | 1ull) >= (worst | 1ull)) guess = KEY_EMPTY;
+        const uint64_t nxt = next_pos < ef_s ? pool[next_pos] : KEY_EMPTY;
+        if ((nxt | 1ull) < (guess | 1ull)) guess = nxt;
+        if (guess != KEY_EMPTY) {
+            const char* p0 = reinterpret_cast<const char*>(enc_hot + (size_t)key_rank(guess) * enc_stride);
+            const char* line = reinterpret_cast<const char*>(reinterpret_cast<uintptr_t>(p0) & ~(uintptr_t)127) + 128 * lane;
+            if (lane < 3 && line < p0 + enc_bytes) FROG_PREFETCH_FN(line);
+        }
+    }
+#endif
+    return (int)merge_batch<EPL>(pool, key, ef_s, lane);
 }
 
 template <int EPL, int MODE, bool BITMAP>
@@ -169,9 +197,13 @@ frog_search_kernel(const FrogSearchArgs A) {
 
         // distance + merge call; in profile builds the time is split at the end of the distances
         long long t_split = 0;
+        const uint32_t* enc_hot_base = nullptr;   // ENC rows from L_start on (set once the hotspot is known)
+        int enc_hot_bytes = 0;                    // bytes of the first two chunks of a vertex's hotspot
+        int second_pos = NO_POS;                  // pool position of the next unexpanded entry after `first`
         auto EVAL = [&](int ns_, uint32_t flag_) {
             int f_ = evaluate_and_merge<EPL>(A.vectors, A.d_pad, A.ef_s, S.pool, S.cand, S.bar, S.q, S.stage, ns_,
-                                             flag_, !BITMAP, MODE == MODE_PROFILE ? &t_split : nullptr);
+                                             flag_, !BITMAP, enc_hot_base, (size_t)A.H * A.m, enc_hot_bytes, second_pos,
+                                             MODE == MODE_PROFILE ? &t_split : nullptr);
             if (MODE == MODE_PROFILE) {
                 long long n_ = clock64();
                 t_ph[3] += t_split - t_mark;
@@ -240,7 +272,11 @@ frog_search_kernel(const FrogSearchArgs A) {
             }
             FROG_PHASE(0);
             n_dist += ns;
-            int first = EVAL(ns, 0u);
+            enc_hot_base = A.enc + (size_t)L_start * A.m;
+            enc_hot_bytes = min(total, 64) * 4;
+            int packed = EVAL(ns, 0u);
+            int first = packed & 0xFFFF;
+            second_pos = (packed >> 16) & 0xFFFF;
             // lines 7-17
             while (first < A.ef_s) {
                 if ((int)n_exp >= A.max_iters) { st |= FROG_ST_ITER_CAP; break; }
@@ -260,29 +296,48 @@ frog_search_kernel(const FrogSearchArgs A) {
                 ns = 0;
                 for (int c0 = 0; c0 < total && cnt < A.B; c0 += 64) {
                     uint32_t v0 = BOT, v1 = BOT;
-                    if (c0 + lane < total) v0 = ldg_stream_u32(hot + c0 + lane);
-                    if (c0 + 32 + lane < total) v1 = ldg_stream_u32(hot + c0 + 32 + lane);
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        if (half == 1 && (cnt >= A.B || c0 + 32 >= total)) break;
-                        const uint32_t v = half ? v1 : v0;
-                        const bool pred = (v - (uint32_t)l_q) <= span;
-                        const uint32_t M = __ballot_sync(FULL, pred);
-                        const int a = min(__popc(M), A.B - cnt);
-                        const bool admitted = pred && (__popc(M & lt_mask) < a);
-                        if (MODE == MODE_TRACE) {
-                            if (rec_ok && admitted) trace_row[3 + trace_len + cnt + __popc(M & lt_mask)] = v;
-                        }
-                        FROG_PHASE(1);
-                        bool keep = admitted;
-                        if (keep) keep = visited_test_and_set<BITMAP>(S, bitmap, A.hash_bits, v, forgets);
-                        const uint32_t K = __ballot_sync(FULL, keep);
-                        if (keep) S.cand[ns + __popc(K & lt_mask)] = v;
-                        ns += __popc(K);
-                        cnt += a;
-                        scanned = min(total, c0 + 32 * (half + 1));
-                        FROG_PHASE(2);
+                    if (c0 + lane < total) v0 = FROG_ENC_LD(hot + c0 + lane);
+                    if (c0 + 32 + lane < total) v1 = FROG_ENC_LD(hot + c0 + 32 + lane);
+                    // first chunk
+                    const bool pred0 = (v0 - (uint32_t)l_q) <= span;
+                    const uint32_t M0 = __ballot_sync(FULL, pred0);
+                    const int a0 = min(__popc(M0), A.B - cnt);
+                    const int rank0 = __popc(M0 & lt_mask);
+                    const bool adm0 = pred0 && rank0 < a0;
+                    // second chunk: scanned only if budget is left after the first
+                    const int rem = A.B - cnt - a0;
+                    const bool has1 = (c0 + 32 < total) && rem > 0;
+                    const bool pred1 = has1 && ((v1 - (uint32_t)l_q) <= span);
+                    const uint32_t M1 = __ballot_sync(FULL, pred1);
+                    const int a1 = min(__popc(M1), rem);
+                    const int rank1 = __popc(M1 & lt_mask);
+                    const bool adm1 = pred1 && rank1 < a1;
+                    if (MODE == MODE_TRACE && rec_ok) {
+                        if (adm0) trace_row[3 + trace_len + cnt + rank0] = v0;
+                        if (adm1) trace_row[3 + trace_len + cnt + a0 + rank1] = v1;
                     }
+                    FROG_PHASE(1);
+                    // visited check of both chunks; with the bitmap the two atomics are in flight together
+                    bool keep0, keep1;
+                    if (BITMAP) {
+                        const uint32_t bit0 = 1u << (v0 & 31), bit1 = 1u << (v1 & 31);
+                        uint32_t old0 = 0xFFFFFFFFu, old1 = 0xFFFFFFFFu;
+                        if (adm0) old0 = atomicOr(bitmap + (v0 >> 5), bit0);
+                        if (adm1) old1 = atomicOr(bitmap + (v1 >> 5), bit1);
+                        keep0 = (old0 & bit0) == 0;
+                        keep1 = (old1 & bit1) == 0;
+                    } else {
+                        keep0 = adm0 && visited_insert(S.hash, A.hash_bits, v0, forgets);
+                        keep1 = adm1 && visited_insert(S.hash, A.hash_bits, v1, forgets);
+                    }
+                    const uint32_t K0 = __ballot_sync(FULL, keep0);
+                    const uint32_t K1 = __ballot_sync(FULL, keep1);
+                    if (keep0) S.cand[ns + __popc(K0 & lt_mask)] = v0;
+                    if (keep1) S.cand[ns + __popc(K0) + __popc(K1 & lt_mask)] = v1;
+                    ns += __popc(K0) + __popc(K1);
+                    cnt += a0 + a1;
+                    scanned = min(total, c0 + (has1 ? 64 : 32));
+                    FROG_PHASE(2);
                 }
                 __syncwarp();
                 ++n_exp;
@@ -297,7 +352,9 @@ frog_search_kernel(const FrogSearchArgs A) {
                         trace_ok = false;
                     }
                 }
-                first = EVAL(ns, 0u);   // lines 14-17
+                packed = EVAL(ns, 0u);   // lines 14-17
+                first = packed & 0xFFFF;
+                second_pos = (packed >> 16) & 0xFFFF;
             }
         }
 
