@@ -67,7 +67,8 @@ typedef struct {
     uint64_t seed;      /* seed of the entry-point generator */
     int32_t hash_bits;  /* FROG_VISITED_HASH: log2 of the table slots; 0 = chosen from beam_width */
     int32_t visited;    /* FROG_VISITED_*: where the visited set lives */
-    int32_t debug_flags;/* bit 0: with `trace`, record per-phase cycle counts instead of EN lists */
+    int32_t debug_flags;/* bit 0: with `trace`, record per-phase cycle counts instead of EN lists;
+                           bit 1: process queries in input order (no heaviest-first planning pass) */
     int32_t reserved;
 } frog_params_t;
 

@@ -49,12 +49,12 @@ int alloc_device(frog_index* ix) {
         (e = cudaMalloc(&ix->d_rank2id, b_attr)) != cudaSuccess ||
         (e = cudaMalloc(&ix->d_vectors, b_vec)) != cudaSuccess ||
         (e = cudaMalloc(&ix->d_enc, b_enc)) != cudaSuccess ||
-        (e = cudaMalloc(&ix->d_work, 256)) != cudaSuccess) {
+        (e = cudaMalloc(&ix->d_work, 1024)) != cudaSuccess) {
         froghost::set_cuda_error(e);
         return e == cudaErrorMemoryAllocation ? FROG_ERR_NOMEM : FROG_ERR_CUDA;
     }
-    ix->info.device_bytes = (int64_t)(2 * b_attr + b_vec + b_enc + 256);
-    FROG_CUDA_TRY(cudaMemset(ix->d_work, 0, 256));
+    ix->info.device_bytes = (int64_t)(2 * b_attr + b_vec + b_enc + 1024);
+    FROG_CUDA_TRY(cudaMemset(ix->d_work, 0, 1024));
     cudaDeviceProp prop;
     FROG_CUDA_TRY(cudaGetDeviceProperties(&prop, I.device));
     ix->sm_count = prop.multiProcessorCount;
@@ -114,6 +114,7 @@ extern "C" void frog_index_free(frog_index_t* ix) {
         cudaFree(ix->d_enc);
         cudaFree(ix->d_work);
         cudaFree(ix->d_bitmap);
+        cudaFree(ix->d_plan);
         cudaFree(ix->d_stage);
     }
     delete ix;

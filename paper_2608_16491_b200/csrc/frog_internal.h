@@ -15,6 +15,8 @@ struct frog_index {
     unsigned int* d_work = nullptr;  // scratch: work counter of the persistent kernel (+ spare words)
     uint32_t* d_bitmap = nullptr;    // scratch: per-warp visited slabs (bitmap_slots x words per slot)
     size_t bitmap_slots = 0;
+    int32_t* d_plan = nullptr;       // scratch: per-query rank interval (2 ints) and processing order (1 int)
+    size_t plan_queries = 0;
     // staging for frog_search_host, grown on demand
     void* d_stage = nullptr;
     size_t stage_bytes = 0;
@@ -42,12 +44,15 @@ struct FrogSearchArgs {
     unsigned int* work_counter;
     uint32_t* bitmap;          // visited slabs, or null when the shared-memory table is used
     size_t bitmap_words;       // words per slab
+    const int2* ranges;        // precomputed [l_q, r_q] per query, or null: computed in the kernel
+    const int32_t* order;      // processing order (heaviest first), or null: input order
 };
 
 namespace froghost {
 void set_cuda_error(cudaError_t e);
 int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in, frog_params_t* out);
 int ensure_bitmap(const frog_index* ix, size_t slots);
+int ensure_plan(const frog_index* ix, size_t nq);
 }  // namespace froghost
 
 #define FROG_CUDA_TRY(expr)                                  \

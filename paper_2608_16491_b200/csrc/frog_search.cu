@@ -180,7 +180,10 @@ frog_search_kernel(const FrogSearchArgs A) {
 
     for (;;) {
         int q = 0;
-        if (lane == 0) q = (int)atomicAdd(A.work_counter, 1u);
+        if (lane == 0) {
+            q = (int)atomicAdd(A.work_counter, 1u);
+            if (q < A.nq && A.order) q = __ldg(A.order + q);
+        }
         q = __shfl_sync(FULL, q, 0);
         if (q >= A.nq) break;
 
@@ -222,7 +225,13 @@ frog_search_kernel(const FrogSearchArgs A) {
         }
         const int32_t lo = __ldg(A.lo + q), hi = __ldg(A.hi + q);
         int l_q, r_q;
-        warp_rank_interval(A.sorted_attr, A.n, lo, hi, lane, l_q, r_q);    // Sec. 4
+        if (A.ranges) {
+            const int2 lr = __ldg(A.ranges + q);
+            l_q = lr.x;
+            r_q = lr.y;
+        } else {
+            warp_rank_interval(A.sorted_attr, A.n, lo, hi, lane, l_q, r_q);    // Sec. 4
+        }
         const int w = (lo > hi) ? 0 : (r_q - l_q + 1);
         uint32_t st = 0, n_exp = 0, n_rows = 0, n_en = 0, n_dist = 0, forgets = 0;
         uint32_t trace_len = 0;
@@ -395,6 +404,44 @@ frog_search_kernel(const FrogSearchArgs A) {
     }
 }
 
+// ---- planning pass: endpoint conversion for the whole batch and a heaviest-first order ---------
+// Queries differ in cost by the width of their range (wider ranges survive the filter more often
+// and evaluate more distances).  With only a few queries per resident warp, the batch ends when the
+// last long query does, so long queries are started first: queries are bucketed by floor(log2 w)
+// and processed bucket by bucket in descending order.
+constexpr int PLAN_HIST = 64, PLAN_CURSOR = 128;   // word offsets in the index's 1 KB work area
+
+__global__ void __launch_bounds__(256)
+frog_plan_kernel(const int32_t* __restrict__ sorted_attr, int n, const int32_t* __restrict__ lo,
+                 const int32_t* __restrict__ hi, int nq, int2* __restrict__ ranges, unsigned int* work) {
+    const int q = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    const int lane = lane_id();
+    if (q >= nq) return;
+    const int32_t lo_q = __ldg(lo + q), hi_q = __ldg(hi + q);
+    int l_q, r_q;
+    warp_rank_interval(sorted_attr, n, lo_q, hi_q, lane, l_q, r_q);        // Sec. 4
+    if (lane == 0) {
+        ranges[q] = make_int2(l_q, r_q);
+        const int w = (lo_q > hi_q) ? 0 : (r_q - l_q + 1);
+        const int bucket = w <= 0 ? 0 : 32 - __clz(w);
+        atomicAdd(work + PLAN_HIST + bucket, 1u);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+frog_order_kernel(const int32_t* __restrict__ lo, const int32_t* __restrict__ hi, int nq,
+                  const int2* __restrict__ ranges, int32_t* __restrict__ order, unsigned int* work) {
+    const int q = (int)(blockIdx.x * blockDim.x + threadIdx.x);
+    if (q >= nq) return;
+    const int2 lr = ranges[q];
+    const int w = (__ldg(lo + q) > __ldg(hi + q)) ? 0 : (lr.y - lr.x + 1);
+    const int bucket = w <= 0 ? 0 : 32 - __clz(w);
+    unsigned int base = 0;
+    for (int b = bucket + 1; b <= 32; ++b) base += work[PLAN_HIST + b];   // queries in heavier buckets
+    const unsigned int pos = base + atomicAdd(work + PLAN_CURSOR + bucket, 1u);
+    order[pos] = q;
+}
+
 typedef void (*kernel_fn)(const FrogSearchArgs);
 
 template <int MODE, bool BITMAP>
@@ -498,6 +545,24 @@ int ensure_bitmap(const frog_index* cix, size_t slots) {
     return FROG_OK;
 }
 
+// Per-query planning scratch: 3 ints per query, grown when a batch is larger than any before.
+int ensure_plan(const frog_index* cix, size_t nq) {
+    frog_index* ix = const_cast<frog_index*>(cix);
+    if (ix->d_plan && ix->plan_queries >= nq) return FROG_OK;
+    FROG_CUDA_TRY(cudaDeviceSynchronize());
+    if (ix->d_plan) FROG_CUDA_TRY(cudaFree(ix->d_plan));
+    ix->d_plan = nullptr;
+    ix->plan_queries = 0;
+    cudaError_t e = cudaMalloc(&ix->d_plan, nq * 3 * sizeof(int32_t));
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        set_cuda_error(e);
+        return FROG_ERR_NOMEM;
+    }
+    ix->plan_queries = nq;
+    return FROG_OK;
+}
+
 }  // namespace froghost
 
 extern "C" int frog_search_launch_info(const frog_index_t* index, int beam_width, const frog_params_t* params,
@@ -576,9 +641,22 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     A.work_counter = index->d_work;
     A.bitmap = bitmap ? index->d_bitmap : nullptr;
     A.bitmap_words = bitmap_words_per_slot(index);
+    A.ranges = nullptr;
+    A.order = nullptr;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    FROG_CUDA_TRY(cudaMemsetAsync(index->d_work, 0, sizeof(unsigned int), s));
+    FROG_CUDA_TRY(cudaMemsetAsync(index->d_work, 0, 1024, s));
+    // planning pass (skipped for tiny batches and when its scratch cannot be had)
+    const bool planned = !(P.debug_flags & 2) && nq >= 64 && froghost::ensure_plan(index, (size_t)nq) == FROG_OK;
+    if (planned) {
+        int2* ranges = reinterpret_cast<int2*>(index->d_plan);
+        int32_t* order = index->d_plan + 2 * (size_t)index->plan_queries;
+        frog_plan_kernel<<<(nq * 32 + 255) / 256, 256, 0, s>>>(index->d_sorted_attr, A.n, lo, hi, nq, ranges,
+                                                               index->d_work);
+        frog_order_kernel<<<(nq + 255) / 256, 256, 0, s>>>(lo, hi, nq, ranges, order, index->d_work);
+        A.ranges = ranges;
+        A.order = order;
+    }
     plan.fn<<<plan.grid, plan.block, plan.smem, s>>>(A);
     FROG_CUDA_TRY(cudaGetLastError());
     return FROG_OK;
@@ -688,6 +766,8 @@ extern "C" int frog_search_static(const frog_index_t* index, const float* querie
     A.work_counter = scratch;                               // word 0 of the header
     A.bitmap = scratch + STATIC_HEADER_WORDS;
     A.bitmap_words = words;
+    A.ranges = nullptr;                                     // endpoints and order are computed in the kernel
+    A.order = nullptr;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the array keeps what the previous call left: the counter must restart at zero; every warp
