@@ -35,6 +35,9 @@ SWEEP = [16, 24, 32, 48, 64, 80, 96, 112, 128, 160, 192, 256, 384, 512]
 BUDGETS = [16, 32]          # expansion budget B of Alg. 2: the paper's default and the kernel's maximum
 RECALL_TARGET = 0.95
 HBM_FALLBACK_GBS = 6650.0
+# DRAM bytes of one search-kernel launch at the default bench point (sift, B = 32, ef_s = 112), from
+# the ncu capture summarised in profiles/frog_search_kernel_sift1m_b32_ef112.md
+NCU_TRAFFIC = {("sift", 1_000_000, 32, 112): 6.653e9}
 
 
 def log(*a):
@@ -88,54 +91,66 @@ def recall_tie_aware(dists: np.ndarray, gt_d: np.ndarray) -> float:
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
+    """SM clock and throttle reasons read through NVML (read-only queries) by a background thread
+    every few milliseconds while the timed region runs."""
 
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40,
+               "sw_thermal_slowdown": 0x20}
 
     def __init__(self, device: int):
-        self.samples = []
-        self.proc = None
+        self.samples = []          # (time, sm_mhz, reasons bitmask)
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "50", "-i", str(device)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
-            self.thread.start()
-        except Exception:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            # NVML enumerates physical devices: honour CUDA_VISIBLE_DEVICES when it lists indices
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            idx = device
+            if vis and all(t.strip().isdigit() for t in vis.split(",")):
+                idx = int(vis.split(",")[device])
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        except Exception as e:           # no NVML: the clocks entry stays empty
+            log(f"[bench] clock sampling unavailable: {e}")
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.samples.append((time.time(), line.strip()))
-
-    def stop(self):
-        if self.proc is not None:
-            self.proc.terminate()
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
             try:
-                self.proc.wait(timeout=5)
+                mhz = float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    rs = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    rs = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                self.samples.append((time.time(), mhz, rs))
             except Exception:
                 pass
+            time.sleep(0.004)
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
 
     def summary(self, t0, t1):
-        rows = [s for t, s in self.samples if t0 <= t <= t1] or [s for _, s in self.samples]
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in rows:
-            f = [x.strip() for x in r.split(",")]
-            try:
-                sm.append(float(f[0]))
-                mx.append(float(f[1]))
-            except Exception:
-                continue
-            for nm, v in zip(names, f[3:7]):
-                if v == "Active":
-                    reasons.add(nm)
-        if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
-                "samples": len(sm)}
+        rows = [s for s in self.samples if t0 <= s[0] <= t1]
+        scope = "timed region"
+        if not rows:
+            rows = [s for s in self.samples if t0 - 0.5 <= s[0] <= t1 + 0.5]
+            scope = "within 0.5 s of the timed region"
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        bits = 0
+        for _, _, r in rows:
+            bits |= r
+        return {"sm_mhz": float(np.median([r[1] for r in rows])), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(k for k, v in self.REASONS.items() if bits & v), "samples": len(rows),
+                "scope": scope}
 
 
 def algorithmic_bytes(stats: np.ndarray, n: int, d: int, d_pad: int, m: int, k: int) -> float:
@@ -365,9 +380,10 @@ def run_ours(args):
         "e2e": {"value": ws * nq * args.steps / e2e_s_max, "unit": UNIT,
                 "h2d_bytes_per_step": nq * info.d * 4 + 2 * nq * 4, "d2h_bytes_per_step": 2 * nq * k * 4,
                 "same_ids_as_device_path": e2e_same},
-        "gpu_launches": args.steps,
+        "gpu_launches": 3 * args.steps,   # per step: endpoint/plan kernel, order kernel, search kernel
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                     "frac": achieved / peak, "peak_source": peak_src,
+                     "traffic": NCU_TRAFFIC.get((wl.name, wl.n, budget, beam)),
                      "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": mean_launch_ms,
                      "kernel": "frog_search_kernel"},
         "clocks": clocks,
