@@ -1,0 +1,103 @@
+"""The bench workload at full size (n = 1,000,000, d = 128, 10,000 queries) in the launch
+configuration bench.py times: sampled queries against the oracle one by one, and properties that
+hold at any size on the whole batch.  Builds the index with the host builder unless a cached
+file exists (about a minute on 16 cores); set FROG_SKIP_FULLSIZE=1 to skip."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+BEAM, BUDGET = 112, 32
+
+
+@pytest.fixture(scope="module")
+def full(libs):
+    if os.environ.get("FROG_SKIP_FULLSIZE") == "1":
+        pytest.skip("FROG_SKIP_FULLSIZE=1")
+    import bench
+    import datagen
+    wl = datagen.make_workload("sift")
+    path, _ = bench.prepare_index(libs, wl, os.environ.get("FROG_CACHE", "/tmp/frog_cache"))
+    gix = libs.Index.load(path, 0)
+    q = torch.from_numpy(wl.queries).cuda()
+    lo = torch.from_numpy(wl.lo).cuda()
+    hi = torch.from_numpy(wl.hi).cuda()
+    status = torch.zeros(wl.nq, dtype=torch.int32, device="cuda")
+    stats = torch.zeros((wl.nq, 4), dtype=torch.int32, device="cuda")
+    ids, dists = gix.search(q, lo, hi, wl.k, BEAM, params=libs.Params(budget=BUDGET), status=status, stats=stats)
+    torch.cuda.synchronize()
+    out = dict(wl=wl, path=path, gix=gix, q=q, lo=lo, hi=hi, ids=ids.cpu().numpy(), dists=dists.cpu().numpy(),
+               status=status.cpu().numpy().view(np.uint32), stats=stats.cpu().numpy().view(np.uint32))
+    yield out
+    gix.close()
+
+
+def test_sampled_queries_equal_the_oracle(full):
+    wl = full["wl"]
+    ix = oracle.load_index(full["path"])
+    rng = np.random.default_rng(7)
+    sample = np.sort(rng.choice(wl.nq, size=400, replace=False))
+    ref = oracle.search(ix, wl.queries[sample], wl.lo[sample], wl.hi[sample], wl.k, BEAM, B=BUDGET)
+    assert np.array_equal(full["ids"][sample], ref.ids)                    # bit-exact ids
+    fin = np.isfinite(ref.dists)
+    assert np.allclose(full["dists"][sample][fin], ref.dists[fin], rtol=1e-4, atol=0)
+    assert np.array_equal(full["dists"][sample][fin], ref.dists[fin])      # same arithmetic order
+    assert np.array_equal(full["status"][sample], ref.status)
+    assert np.array_equal(full["stats"][sample], ref.stats)                # expansions, rows, ENs, distances
+    # recall of the two implementations against exact filtered kNN on the sample
+    gt, _, _ = oracle.exact_slab(ix, wl.queries[sample], wl.lo[sample], wl.hi[sample], wl.k, mode=0)
+    assert abs(oracle.recall(full["ids"][sample], gt) - oracle.recall(ref.ids, gt)) <= 0.005
+    assert oracle.recall(full["ids"][sample], gt) >= 0.93
+
+
+def test_whole_batch_properties(full):
+    wl, ids, dists = full["wl"], full["ids"], full["dists"]
+    valid = ids >= 0
+    # every result satisfies lo <= attr <= hi
+    a = wl.attrs[np.where(valid, ids, 0)]
+    assert np.all(~valid | ((a >= wl.lo[:, None]) & (a <= wl.hi[:, None])))
+    # ascending distances, padding only at the tail, no repeated id in a row
+    assert np.all(np.diff(np.where(valid, dists, np.inf), axis=1) >= 0)
+    assert np.all(valid[:, :-1] | ~valid[:, 1:])
+    srt = np.sort(np.where(valid, ids, -np.arange(1, ids.shape[1] + 1)[None, :]), axis=1)
+    assert np.all(np.diff(srt, axis=1) != 0)
+    # reported distances are the true ones (integer-valued data: exact in fp32)
+    rows = wl.vectors[np.where(valid, ids, 0)]                              # [nq, k, d]
+    true = np.sqrt(((rows.astype(np.float64) - wl.queries[:, None, :].astype(np.float64)) ** 2).sum(-1))
+    assert np.allclose(dists[valid], true[valid], rtol=1e-6)
+    # small ranges were answered exactly and never flagged otherwise
+    st = full["status"]
+    assert not (st & 4).any() and not (st & 32).any()                       # no iteration cap, no copy timeout
+
+
+def test_exact_search_at_full_size_on_sampled_queries(full, libs):
+    wl = full["wl"]
+    ix = oracle.load_index(full["path"])
+    ids, dists = full["gix"].exact_search(full["q"], full["lo"], full["hi"], wl.k)
+    torch.cuda.synchronize()
+    ids, dists = ids.cpu().numpy(), dists.cpu().numpy()
+    rng = np.random.default_rng(11)
+    sample = np.sort(rng.choice(wl.nq, size=60, replace=False))
+    ref_ids, ref_d, _ = oracle.exact_slab(ix, wl.queries[sample], wl.lo[sample], wl.hi[sample], wl.k, mode=1)
+    assert np.array_equal(ids[sample], ref_ids) and np.array_equal(dists[sample], ref_d)
+    # against the definition scan over raw (vectors, attrs): equal up to exact distance ties
+    def_ids, def_d = oracle.exact_scan(wl.vectors, wl.attrs, wl.queries[sample[:12]], wl.lo[sample[:12]],
+                                       wl.hi[sample[:12]], wl.k, mode=0)
+    assert np.allclose(dists[sample[:12]], def_d, rtol=1e-6)
+
+
+def test_static_entry_point_at_full_size(full, libs):
+    """The allocation-free entry point on the 1M index (fewer resident warps, same answers)."""
+    wl = full["wl"]
+    out_ids = torch.empty((wl.nq, wl.k), dtype=torch.int32, device="cuda")
+    out_d = torch.empty((wl.nq, wl.k), dtype=torch.float32, device="cuda")
+    full["gix"].search_static(full["q"], full["lo"], full["hi"], wl.k, BEAM, out_ids=out_ids, out_dists=out_d,
+                              params=libs.Params(budget=BUDGET))
+    torch.cuda.synchronize()
+    assert np.array_equal(out_ids.cpu().numpy(), full["ids"])
