@@ -53,20 +53,32 @@ def measured_hbm_peak():
         return HBM_FALLBACK_GBS, "fallback"
 
 
-def prepare_index(frog, wl, cache_dir):
-    """Build (or reuse) the index file of a workload.  The cache is an optimisation only."""
+def prepare_index(frog, wl, cache_dir, builder="auto", device=0):
+    """Build (or reuse) the index file of a workload.  The cache is an optimisation only.
+    builder: "gpu" (CUDA builder), "cpu" (host builder) or "auto" (gpu when a device is there)."""
     os.makedirs(cache_dir, exist_ok=True)
     from paper_2608_16491_b200 import build as b
+    if builder == "auto":
+        try:
+            import torch
+            builder = "gpu" if torch.cuda.is_available() else "cpu"
+        except Exception:
+            builder = "cpu"
+    src = "frog_build_gpu.cu" if builder == "gpu" else "frog_build.cpp"
     h = hashlib.sha1()
-    h.update(open(os.path.join(b.CSRC, "frog_build.cpp"), "rb").read())
+    h.update(open(os.path.join(b.CSRC, src), "rb").read())
+    h.update(open(os.path.join(b.CSRC, "frog_device.cuh"), "rb").read() if builder == "gpu" else b"")
     h.update(open(os.path.join(ROOT, "datagen", "__init__.py"), "rb").read())
     tag = h.hexdigest()[:12]
-    path = os.path.join(cache_dir, f"{wl.name}_{wl.n}_{tag}.idx")
+    path = os.path.join(cache_dir, f"{wl.name}_{wl.n}_{builder}_{tag}.idx")
     secs = 0.0
     if not os.path.exists(path):
         t = time.time()
         tmp = path + f".tmp{os.getpid()}"
-        frog.build_index(wl.vectors, wl.attrs, tmp, seed=wl.seed)
+        if builder == "gpu":
+            frog.build_index_gpu(wl.vectors, wl.attrs, tmp, device=device, seed=wl.seed)
+        else:
+            frog.build_index(wl.vectors, wl.attrs, tmp, seed=wl.seed)
         os.replace(tmp, path)
         secs = time.time() - t
     return path, secs
@@ -186,7 +198,7 @@ def run_reference(args):
     import oracle
     import paper_2608_16491_b200 as frog
     wl = datagen.make_workload(args.workload, n=args.n or None, nq=args.nq or None)
-    path, build_s = prepare_index(frog, wl, args.cache_dir)
+    path, build_s = prepare_index(frog, wl, args.cache_dir, args.builder)
     ix = oracle.load_index(path)
     S = min(args.ref_sample, wl.nq)
     Q, lo, hi = wl.queries[:S], wl.lo[:S], wl.hi[:S]
@@ -240,10 +252,10 @@ def run_ours(args):
     wl = datagen.make_workload(args.workload, n=args.n or None, nq=args.nq or None)
     gen_s = time.time() - t
     if rank == 0:
-        path, build_s = prepare_index(frog, wl, args.cache_dir)
+        path, build_s = prepare_index(frog, wl, args.cache_dir, args.builder, local_rank)
     replicas.barrier()
     if rank != 0:
-        path, build_s = prepare_index(frog, wl, args.cache_dir)
+        path, build_s = prepare_index(frog, wl, args.cache_dir, args.builder, local_rank)
     t = time.time()
     ix = frog.Index.load(path, local_rank)
     load_s = time.time() - t
@@ -373,7 +385,8 @@ def run_ours(args):
                                f"(width fraction log-uniform 2^-10..1)",
                    "beam_width": beam, "recall_at_10": chosen["recall"],
                    "recall_tie_aware": chosen["recall_tie_aware"], "epn": 16, "budget": budget,
-                   "index": {"H": info.H, "m": info.m, "bytes": info.device_bytes, "build_seconds": round(build_s, 1)},
+                   "index": {"H": info.H, "m": info.m, "bytes": info.device_bytes, "build_seconds": round(build_s, 1),
+                             "file": os.path.basename(path)},
                    "l2": "inputs larger than L2 (1.4 GB index, ~%.1f GB gathered per launch)" % (alg_bytes / 1e9),
                    "parallelism": "replicas" if ws > 1 else "single GPU",
                    "launch": launch, "sweep": sweep},
@@ -407,6 +420,8 @@ def main():
     ap.add_argument("--beam", type=int, default=0, help="beam width; 0 = smallest reaching the recall target")
     ap.add_argument("--budget", type=int, default=0, help="expansion budget B; 0 = best of 16 and 32")
     ap.add_argument("--cache-dir", default=os.environ.get("FROG_CACHE", "/tmp/frog_cache"))
+    ap.add_argument("--builder", default="auto", choices=["auto", "gpu", "cpu"],
+                    help="index builder used when the cache has no file for the workload")
     ap.add_argument("--cpu-sample", type=int, default=4000)
     ap.add_argument("--ref-sample", type=int, default=1000)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -111,6 +111,22 @@ def build_index(vectors: np.ndarray, attrs: np.ndarray, path: str, m: int = 0, e
         raise FrogError(rc, "frog_index_build")
 
 
+def build_index_gpu(vectors: np.ndarray, attrs: np.ndarray, path: str, device: int = 0, m: int = 0,
+                    ef_c: int = 0, n_inv: int = -1, patience: int = 0, beta: float = -1.0,
+                    gamma: float = 0.0, seed: int = 0) -> None:
+    """Build the FROG index of (vectors, attrs) with the CUDA builder and write it to ``path``."""
+    v = np.ascontiguousarray(vectors, dtype=np.float32)
+    a = np.ascontiguousarray(attrs, dtype=np.int32)
+    if v.ndim != 2 or a.shape != (v.shape[0],):
+        raise ValueError("vectors must be [n, d] and attrs [n]")
+    p = BuildParams(m=m, ef_c=ef_c, n_inv=n_inv, patience=patience, beta=beta, gamma=gamma,
+                    seed=seed, threads=0, reserved=0)
+    rc = _lib.frog_index_build_gpu(v.ctypes.data_as(_vp), a.ctypes.data_as(_vp), C.c_int64(v.shape[0]),
+                                   C.c_int32(v.shape[1]), C.byref(p), C.c_int(device), path.encode())
+    if rc != 0:
+        raise FrogError(rc, "frog_index_build_gpu")
+
+
 def _ptr(t) -> C.c_void_p:
     return _vp(0) if t is None else _vp(t.data_ptr())
 

@@ -18,7 +18,7 @@ INCLUDE = os.path.join(ROOT, "include")
 LIB_SEARCH = os.path.join(HERE, "libfrog.so")
 LIB_BUILD = os.path.join(HERE, "libfrog_build.so")
 
-CUDA_SOURCES = ["frog_index.cu", "frog_search.cu", "frog_exact.cu"]
+CUDA_SOURCES = ["frog_index.cu", "frog_search.cu", "frog_exact.cu", "frog_build_gpu.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--fmad=false", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

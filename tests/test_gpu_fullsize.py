@@ -1,7 +1,7 @@
 """The bench workload at full size (n = 1,000,000, d = 128, 10,000 queries) in the launch
 configuration bench.py times: sampled queries against the oracle one by one, and properties that
-hold at any size on the whole batch.  Builds the index with the host builder unless a cached
-file exists (about a minute on 16 cores); set FROG_SKIP_FULLSIZE=1 to skip."""
+hold at any size on the whole batch.  Builds the index with the CUDA builder unless a cached
+file exists (a few seconds); set FROG_SKIP_FULLSIZE=1 to skip."""
 import os
 
 import numpy as np
@@ -23,7 +23,7 @@ def full(libs):
     import bench
     import datagen
     wl = datagen.make_workload("sift")
-    path, _ = bench.prepare_index(libs, wl, os.environ.get("FROG_CACHE", "/tmp/frog_cache"))
+    path, _ = bench.prepare_index(libs, wl, os.environ.get("FROG_CACHE", "/tmp/frog_cache"), "gpu")
     gix = libs.Index.load(path, 0)
     q = torch.from_numpy(wl.queries).cuda()
     lo = torch.from_numpy(wl.lo).cuda()
