@@ -101,3 +101,61 @@ def test_static_entry_point_at_full_size(full, libs):
                               params=libs.Params(budget=BUDGET))
     torch.cuda.synchronize()
     assert np.array_equal(out_ids.cpu().numpy(), full["ids"])
+
+
+# ---- the other full-size workloads (opt-in: minutes of generation, building and file I/O) -----------
+ALL = os.environ.get("FROG_FULLSIZE_ALL") == "1"
+
+
+@pytest.mark.skipif(not ALL, reason="set FROG_FULLSIZE_ALL=1 to run the 1M x 96, 10M x 96 and 1M x 768 workloads")
+@pytest.mark.parametrize("name,k,beam", [("deep1m", 10, 128), ("text", 10, 128), ("deep10m", 10, 128),
+                                         ("deep10m", 100, 128)])
+def test_other_workloads_at_full_size(libs, name, k, beam):
+    import bench
+    import datagen
+    wl = datagen.make_workload(name, k=k)
+    path, secs = bench.prepare_index(libs, wl, os.environ.get("FROG_CACHE", "/tmp/frog_cache"), "gpu")
+    gix = libs.Index.load(path, 0)
+    try:
+        q = torch.from_numpy(wl.queries).cuda()
+        lo = torch.from_numpy(wl.lo).cuda()
+        hi = torch.from_numpy(wl.hi).cuda()
+        status = torch.zeros(wl.nq, dtype=torch.int32, device="cuda")
+        stats = torch.zeros((wl.nq, 4), dtype=torch.int32, device="cuda")
+        prm = libs.Params(budget=BUDGET)
+        ids, dists = gix.search(q, lo, hi, k, beam, params=prm, status=status, stats=stats)
+        torch.cuda.synchronize()
+        ids, dists = ids.cpu().numpy(), dists.cpu().numpy()
+        st = status.cpu().numpy().view(np.uint32)
+        # sampled queries, one by one, against the oracle on the same index file
+        ix = oracle.load_index(path)
+        rng = np.random.default_rng(5)
+        sample = np.sort(rng.choice(wl.nq, size=200, replace=False))
+        ref = oracle.search(ix, wl.queries[sample], wl.lo[sample], wl.hi[sample], k, beam, B=BUDGET)
+        assert np.array_equal(ids[sample], ref.ids)
+        fin = np.isfinite(ref.dists)
+        assert np.allclose(dists[sample][fin], ref.dists[fin], rtol=1e-4, atol=0)
+        assert np.array_equal(st[sample], ref.status)
+        assert np.array_equal(stats.cpu().numpy().view(np.uint32)[sample], ref.stats)
+        gt, _, _ = oracle.exact_slab(ix, wl.queries[sample], wl.lo[sample], wl.hi[sample], k, mode=0)
+        rec_gpu, rec_ref = oracle.recall(ids[sample], gt), oracle.recall(ref.ids, gt)
+        assert abs(rec_gpu - rec_ref) <= 0.005
+        print(f"[fullsize] {name} k={k} beam={beam}: build {secs:.1f}s recall@{k} {rec_gpu:.4f} (sample of 200)")
+        # whole batch: range, order, padding
+        valid = ids >= 0
+        a = wl.attrs[np.where(valid, ids, 0)]
+        assert np.all(~valid | ((a >= wl.lo[:, None]) & (a <= wl.hi[:, None])))
+        assert np.all(np.diff(np.where(valid, dists, np.inf), axis=1) >= 0)
+        assert np.all(valid[:, :-1] | ~valid[:, 1:])
+        assert not (st & 4).any() and not (st & 32).any()
+        # exact search on a few queries of the sample
+        e_ids, e_d = gix.exact_search(q[:64], lo[:64], hi[:64], k)
+        torch.cuda.synchronize()
+        r_ids, r_d, _ = oracle.exact_slab(ix, wl.queries[:64], wl.lo[:64], wl.hi[:64], k, mode=1)
+        assert np.array_equal(e_ids.cpu().numpy(), r_ids) and np.array_equal(e_d.cpu().numpy(), r_d)
+    finally:
+        gix.close()
+        # do not leave multi-gigabyte files behind on a shared machine (the 10M index is reused by the
+        # k = 100 case that follows it in the parameter list)
+        if os.path.getsize(path) > (4 << 30) and not (name == "deep10m" and k == 10):
+            os.remove(path)
