@@ -777,3 +777,4 @@ extern "C" int frog_search_static(const frog_index_t* index, const float* querie
     FROG_CUDA_TRY(cudaGetLastError());
     return FROG_OK;
 }
+
