@@ -372,7 +372,7 @@ int frog_oracle_search(const int32_t* sorted_attr, const int32_t* rank2id, const
     Params P{epn, B, max_iters, seed, warp, no_hotspot};
     int used = 1;
 #ifdef _OPENMP
-    if (threads > 0) omp_set_num_threads(threads);
+    omp_set_num_threads(threads > 0 ? threads : omp_get_num_procs());   // <= 0: all cores
     used = omp_get_max_threads();
 #endif
 #pragma omp parallel for schedule(dynamic, 4)
@@ -401,7 +401,7 @@ int frog_oracle_exact_scan(const float* vectors, const int32_t* attrs, int64_t n
                            int k, int mode, int32_t* out_ids, float* out_dists, int threads) {
     int used = 1;
 #ifdef _OPENMP
-    if (threads > 0) omp_set_num_threads(threads);
+    omp_set_num_threads(threads > 0 ? threads : omp_get_num_procs());   // <= 0: all cores
     used = omp_get_max_threads();
 #endif
 #pragma omp parallel for schedule(dynamic, 1)
@@ -436,7 +436,7 @@ int frog_oracle_exact_slab(const int32_t* sorted_attr, const int32_t* rank2id, c
                            int k, int mode, int32_t* out_ids, float* out_dists, int threads) {
     int used = 1;
 #ifdef _OPENMP
-    if (threads > 0) omp_set_num_threads(threads);
+    omp_set_num_threads(threads > 0 ? threads : omp_get_num_procs());   // <= 0: all cores
     used = omp_get_max_threads();
 #endif
 #pragma omp parallel for schedule(dynamic, 1)
