@@ -67,10 +67,17 @@ typedef struct {
     uint64_t seed;      /* seed of the entry-point generator */
     int32_t hash_bits;  /* FROG_VISITED_HASH: log2 of the table slots; 0 = chosen from beam_width */
     int32_t visited;    /* FROG_VISITED_*: where the visited set lives */
+    int32_t storage;    /* FROG_STORAGE_*: which copy of the vectors the gather reads */
     int32_t debug_flags;/* bit 0: with `trace`, record per-phase cycle counts instead of EN lists;
                            bit 1: process queries in input order (no heaviest-first planning pass) */
-    int32_t reserved;
 } frog_params_t;
+
+/* Vector storage read by the search.  F32 (default): the index's fp32 rows.  F16: an fp16 copy made
+ * by frog_index_enable_f16 (half the gathered bytes; values are converted back to fp32 and all
+ * arithmetic stays fp32, so the result equals a search over the fp16-rounded vectors exactly; the
+ * paper's own GPU programs read float16 data, Sec. 8.1.4).  F16 needs the bitmap visited form. */
+#define FROG_STORAGE_F32 0
+#define FROG_STORAGE_F16 1
 
 /* Visited set (hashCheck of Alg. 2).  BITMAP: one bit per rank in a per-warp slab of device
  * scratch memory owned by the index (n/8 bytes per resident warp, allocated on first use, exact).
@@ -106,6 +113,11 @@ int frog_index_from_host(const int32_t* sorted_attr, const int32_t* rank2id, con
 void frog_index_free(frog_index_t* index);
 
 int frog_index_info(const frog_index_t* index, frog_index_info_t* out);
+
+/* frog_index_enable_f16: add an fp16 copy of the vectors to the index (round to nearest even,
+ * rows padded to a multiple of 8 elements; n * 2 * 8 * ceil(d / 8) more bytes of device memory).
+ * Idempotent.  Searches select it with params->storage = FROG_STORAGE_F16. */
+int frog_index_enable_f16(frog_index_t* index);
 
 /* frog_search: batched FROGSearch (Alg. 2, with Alg. 3 once per query and Alg. 4 plus the lazy
  * hash check of Sec. 7.3.2 at every expansion), one query per warp of a persistent kernel.

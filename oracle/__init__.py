@@ -100,6 +100,14 @@ def load_index(path: str) -> OracleIndex:
         enc=arr(o_enc, n * H * m, np.uint32).reshape(n, H, m))
 
 
+def rounded_to_f16(ix: OracleIndex) -> OracleIndex:
+    """The same index with every vector component rounded to the nearest fp16 value (ties to even)
+    and widened back to fp32: what a search over half-precision storage sees.  Arithmetic is
+    unchanged (fp32, same order), only the stored values differ."""
+    v = np.asarray(ix.vectors).astype(np.float16).astype(np.float32)
+    return dataclasses.replace(ix, vectors=np.ascontiguousarray(v))
+
+
 def pad_queries(queries: np.ndarray, d_pad: int) -> np.ndarray:
     q = np.ascontiguousarray(queries, dtype=np.float32)
     if q.shape[1] == d_pad:

@@ -26,6 +26,7 @@ _LIB_BUILD = os.path.join(_HERE, "libfrog_build.so")
 FROG_MAX_BEAM_WIDTH = 512
 ST_EMPTY, ST_EXACT, ST_ITER_CAP, ST_SHORT, ST_FORGOT = 1, 2, 4, 8, 16
 VISITED_AUTO, VISITED_BITMAP, VISITED_HASH = 0, 1, 2
+STORAGE_F32, STORAGE_F16 = 0, 1
 
 
 class FrogError(RuntimeError):
@@ -44,7 +45,7 @@ class IndexInfo(C.Structure):
 class Params(C.Structure):
     _fields_ = [("epn", C.c_int32), ("budget", C.c_int32), ("max_iters", C.c_int32),
                 ("no_hotspot", C.c_int32), ("seed", C.c_uint64), ("hash_bits", C.c_int32),
-                ("visited", C.c_int32), ("debug_flags", C.c_int32), ("reserved", C.c_int32)]
+                ("visited", C.c_int32), ("storage", C.c_int32), ("debug_flags", C.c_int32)]
 
 
 class BuildParams(C.Structure):
@@ -155,6 +156,12 @@ class Index:
         if rc:
             raise FrogError(rc, "frog_index_load")
         return cls(h)
+
+    def enable_f16(self) -> None:
+        """Add an fp16 copy of the vectors; searches read it with ``Params(storage=STORAGE_F16)``."""
+        rc = _lib.frog_index_enable_f16(self._h)
+        if rc:
+            raise FrogError(rc, "frog_index_enable_f16")
 
     def close(self) -> None:
         if self._h:

@@ -10,6 +10,7 @@
 #pragma once
 
 #include <cstdint>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 namespace frogdev {
@@ -300,6 +301,78 @@ __device__ __forceinline__ float staged_dist2(const float* __restrict__ vectors,
                 a = a + __shfl_xor_sync(FULL, a, 2);
                 a = a + __shfl_xor_sync(FULL, a, 1);
                 // the result for row r0 + i*4 + t sits in team t; hand it to lane r0 + i*4 + t
+                const float v = __shfl_sync(FULL, a, src);
+                if (lane >= r0 && ((lane - r0) >> 2) == i && lane - r0 < nrows) out = v;
+            }
+        }
+    }
+    return out;
+}
+
+// The same gather + distance with a run-time stage geometry and optional half-precision storage.
+// `rows` points at row-major data of `row_bytes` per row (fp32, or fp16 when F16); a row occupies a
+// slot of `slot_bytes` (>= the chunk, at most STAGE_CHUNK) in the stage buffer and up to
+// `rows_per_pass` (<= 16, multiple of 4) rows complete on one mbarrier phase.  fp16 elements are
+// converted to fp32 on the way out of shared memory; products and sums are fp32 in the same fixed
+// order, so the result equals the fp32 routine run on the rounded values bit for bit.
+template <bool F16>
+__device__ __forceinline__ float staged_dist2_flex(const void* __restrict__ rows, int row_bytes, int slot_bytes,
+                                                   int rows_per_pass, const float4* qs, float4* stage, uint64_t* bar,
+                                                   uint32_t& phase, bool& ok, uint32_t my_rank, int ns, int lane) {
+    const int team = lane >> 3, sub = lane & 7;
+    constexpr int GROUP_BYTES = F16 ? 8 : 16;             // 4 elements
+    float out = 0.f;
+    const int src = (lane & 3) << 3;
+#pragma unroll 1
+    for (int r0 = 0; r0 < ns; r0 += rows_per_pass) {
+        const int nrows = min(rows_per_pass, ns - r0);
+        const uint32_t copy_rank = __shfl_sync(FULL, my_rank, (r0 + lane) & 31);
+        const char* src_row = reinterpret_cast<const char*>(rows) + (size_t)copy_rank * (size_t)row_bytes;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+        for (int c0 = 0; c0 < row_bytes; c0 += STAGE_CHUNK) {
+            const int cbytes = min(STAGE_CHUNK, row_bytes - c0);
+            __syncwarp();                                   // every lane is done reading the stage buffer
+            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(nrows * cbytes));
+            __syncwarp();
+            if (lane < nrows)
+                tma_load_1d(reinterpret_cast<char*>(stage) + lane * slot_bytes, src_row + c0, (uint32_t)cbytes, bar);
+            ok = mbar_wait(bar, phase) && ok;
+            phase ^= 1u;
+            const int g_lo = c0 / GROUP_BYTES, g_n = cbytes / GROUP_BYTES;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = i * 4 + team;
+                if (i * 4 < nrows && r < nrows) {
+                    const char* xrow = reinterpret_cast<const char*>(stage) + r * slot_bytes;
+#pragma unroll 4
+                    for (int g = sub; g < g_n; g += 8) {
+                        float4 x;
+                        if (F16) {
+                            const uint2 raw = *reinterpret_cast<const uint2*>(xrow + g * 8);
+                            const float2 lo2 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+                            const float2 hi2 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+                            x = make_float4(lo2.x, lo2.y, hi2.x, hi2.y);
+                        } else {
+                            x = *reinterpret_cast<const float4*>(xrow + g * 16);
+                        }
+                        const float4 q = qs[g_lo + g];
+                        float t;
+                        t = x.x - q.x; acc[i] = fmaf(t, t, acc[i]);
+                        t = x.y - q.y; acc[i] = fmaf(t, t, acc[i]);
+                        t = x.z - q.z; acc[i] = fmaf(t, t, acc[i]);
+                        t = x.w - q.w; acc[i] = fmaf(t, t, acc[i]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (i * 4 < nrows) {
+                float a = acc[i];
+                a = a + __shfl_xor_sync(FULL, a, 4);
+                a = a + __shfl_xor_sync(FULL, a, 2);
+                a = a + __shfl_xor_sync(FULL, a, 1);
                 const float v = __shfl_sync(FULL, a, src);
                 if (lane >= r0 && ((lane - r0) >> 2) == i && lane - r0 < nrows) out = v;
             }

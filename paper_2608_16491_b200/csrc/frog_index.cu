@@ -111,6 +111,7 @@ extern "C" void frog_index_free(frog_index_t* ix) {
         cudaFree(ix->d_sorted_attr);
         cudaFree(ix->d_rank2id);
         cudaFree(ix->d_vectors);
+        cudaFree(ix->d_vectors_h);
         cudaFree(ix->d_enc);
         cudaFree(ix->d_work);
         cudaFree(ix->d_bitmap);

@@ -11,6 +11,7 @@ struct frog_index {
     int32_t* d_sorted_attr = nullptr;
     int32_t* d_rank2id = nullptr;
     float* d_vectors = nullptr;      // n x d_pad, rank order
+    void* d_vectors_h = nullptr;     // optional fp16 copy, n x d_pad_h (d_pad_h = 8 * ceil(d / 8))
     uint32_t* d_enc = nullptr;       // n x H x m
     unsigned int* d_work = nullptr;  // scratch: work counter of the persistent kernel (+ spare words)
     uint32_t* d_bitmap = nullptr;    // scratch: per-warp visited slabs (bitmap_slots x words per slot)
@@ -46,6 +47,11 @@ struct FrogSearchArgs {
     size_t bitmap_words;       // words per slab
     const int2* ranges;        // precomputed [l_q, r_q] per query, or null: computed in the kernel
     const int32_t* order;      // processing order (heaviest first), or null: input order
+    const void* rows;          // gather source: fp32 vectors, or their fp16 copy
+    int row_bytes;             // bytes per stored row
+    int slot_bytes;            // bytes of one row slot in the stage buffer (power of two, <= 512)
+    int rows_per_pass;         // rows completing on one mbarrier phase (4..16)
+    int q_len;                 // floats of the query held in shared memory (8 * ceil(d / 8))
 };
 
 namespace froghost {

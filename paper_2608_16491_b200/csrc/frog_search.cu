@@ -61,10 +61,11 @@ struct WarpSmem {
     uint32_t* hash;
 };
 
-inline size_t warp_smem_bytes(int pool_slots, int d_pad, int hash_bits, bool bitmap) {
-    return (size_t)pool_slots * 8 + 32 * 4 + 16 + (size_t)d_pad * 4 + STAGE_BYTES +
+inline size_t warp_smem_bytes(int pool_slots, int q_len, int hash_bits, bool bitmap) {
+    return (size_t)pool_slots * 8 + 32 * 4 + 16 + (size_t)q_len * 4 + STAGE_BYTES +
            (bitmap ? 0 : ((size_t)4 << hash_bits));
 }
+inline int query_len(int d) { return (d + 7) / 8 * 8; }
 
 // entry point j of a query range: stateless mixer of (seed, l_q, r_q, j), top 32 bits scaled
 // into [0, w) by a multiply-high (Alg. 2 line 3: uniform sample from [l_q, r_q])
@@ -94,8 +95,9 @@ __device__ __forceinline__ bool visited_test_and_set(const WarpSmem& S, uint32_t
 // Distances of the ns <= 32 ranks listed in cand[0..ns) and their merge into the pool (Alg. 2
 // lines 14-17).  Returns the first unexpanded pool position.  Kept out of line: it is called from
 // three places of the kernel and inlining every copy costs registers and instruction cache.
-template <int EPL>
-__device__ FROG_EVAL_INLINE int evaluate_and_merge(const float* __restrict__ vectors, int d_pad, int ef_s,
+template <int EPL, bool F16>
+__device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows, int row_bytes, int slot_bytes,
+                                                   int rows_per_pass, int ef_s,
                                                    uint64_t* pool, const uint32_t* cand, uint64_t* bar,
                                                    const float4* qs, float4* stage,
                                                    int ns, uint32_t new_flag, bool dedupe,
@@ -123,7 +125,7 @@ __device__ FROG_EVAL_INLINE int evaluate_and_merge(const float* __restrict__ vec
         __syncwarp();                       // lane 0's update of the parity in the previous call
         uint32_t phase = bar_words[0];
         bool ok = true;
-        d2 = staged_dist2<FROG_STAGE_ROWS>(vectors, d_pad, qs, stage, bar, phase, ok, id, ns, lane);
+        d2 = staged_dist2_flex<F16>(rows, row_bytes, slot_bytes, rows_per_pass, qs, stage, bar, phase, ok, id, ns, lane);
         __syncwarp();                       // every lane has read the old parity
         if (lane == 0) {
             bar_words[0] = phase;
@@ -152,7 +154,7 @@ __device__ FROG_EVAL_INLINE int evaluate_and_merge(const float* __restrict__ vec
     return (int)merge_batch<EPL>(pool, key, ef_s, lane);
 }
 
-template <int EPL, int MODE, bool BITMAP>
+template <int EPL, int MODE, bool BITMAP, bool F16>
 __global__ void __launch_bounds__(WARPS_PER_CTA * 32, MODE == MODE_FAST ? (EPL <= 4 ? FROG_MINB : 4) : 1)
 frog_search_kernel(const FrogSearchArgs A) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -160,14 +162,14 @@ frog_search_kernel(const FrogSearchArgs A) {
     const int warp = threadIdx.x >> 5;
     constexpr int POOL = 32 * EPL;
     const int hash_slots = BITMAP ? 0 : (1 << A.hash_bits);
-    const size_t per_warp = (size_t)POOL * 8 + 32 * 4 + 16 + (size_t)A.d_pad * 4 + STAGE_BYTES + (size_t)hash_slots * 4;
+    const size_t per_warp = (size_t)POOL * 8 + 32 * 4 + 16 + (size_t)A.q_len * 4 + STAGE_BYTES + (size_t)hash_slots * 4;
     unsigned char* base = smem_raw + per_warp * warp;
     WarpSmem S;
     S.pool = reinterpret_cast<uint64_t*>(base);
     S.cand = reinterpret_cast<uint32_t*>(S.pool + POOL);
     S.bar = reinterpret_cast<uint64_t*>(S.cand + 32);
     S.q = reinterpret_cast<float4*>(S.bar + 2);
-    S.stage = reinterpret_cast<float4*>(reinterpret_cast<float*>(S.q) + A.d_pad);
+    S.stage = reinterpret_cast<float4*>(reinterpret_cast<float*>(S.q) + A.q_len);
     S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(S.stage) + STAGE_BYTES);
     if (lane == 0) {
         mbar_init(S.bar, 1u);
@@ -204,9 +206,10 @@ frog_search_kernel(const FrogSearchArgs A) {
         int enc_hot_bytes = 0;                    // bytes of the first two chunks of a vertex's hotspot
         int second_pos = NO_POS;                  // pool position of the next unexpanded entry after `first`
         auto EVAL = [&](int ns_, uint32_t flag_) {
-            int f_ = evaluate_and_merge<EPL>(A.vectors, A.d_pad, A.ef_s, S.pool, S.cand, S.bar, S.q, S.stage, ns_,
-                                             flag_, !BITMAP, enc_hot_base, (size_t)A.H * A.m, enc_hot_bytes, second_pos,
-                                             MODE == MODE_PROFILE ? &t_split : nullptr);
+            int f_ = evaluate_and_merge<EPL, F16>(A.rows, A.row_bytes, A.slot_bytes, A.rows_per_pass, A.ef_s, S.pool,
+                                                  S.cand, S.bar, S.q, S.stage, ns_, flag_, !BITMAP, enc_hot_base,
+                                                  (size_t)A.H * A.m, enc_hot_bytes, second_pos,
+                                                  MODE == MODE_PROFILE ? &t_split : nullptr);
             if (MODE == MODE_PROFILE) {
                 long long n_ = clock64();
                 t_ph[3] += t_split - t_mark;
@@ -220,7 +223,7 @@ frog_search_kernel(const FrogSearchArgs A) {
         {
             float* qf = reinterpret_cast<float*>(S.q);
             const float* src = A.queries + (size_t)q * A.d;
-            for (int i = lane; i < A.d_pad; i += 32) qf[i] = i < A.d ? __ldg(src + i) : 0.f;
+            for (int i = lane; i < A.q_len; i += 32) qf[i] = i < A.d ? __ldg(src + i) : 0.f;
             for (int i = lane; i < POOL; i += 32) S.pool[i] = KEY_EMPTY;
         }
         const int32_t lo = __ldg(A.lo + q), hi = __ldg(A.hi + q);
@@ -444,14 +447,14 @@ frog_order_kernel(const int32_t* __restrict__ lo, const int32_t* __restrict__ hi
 
 typedef void (*kernel_fn)(const FrogSearchArgs);
 
-template <int MODE, bool BITMAP>
+template <int MODE, bool BITMAP, bool F16>
 kernel_fn pick_kernel(int ef_s, int* pool_slots) {
-    if (ef_s <= 32) { *pool_slots = 32; return frog_search_kernel<1, MODE, BITMAP>; }
-    if (ef_s <= 64) { *pool_slots = 64; return frog_search_kernel<2, MODE, BITMAP>; }
-    if (ef_s <= 128) { *pool_slots = 128; return frog_search_kernel<4, MODE, BITMAP>; }
-    if (ef_s <= 256) { *pool_slots = 256; return frog_search_kernel<8, MODE, BITMAP>; }
+    if (ef_s <= 32) { *pool_slots = 32; return frog_search_kernel<1, MODE, BITMAP, F16>; }
+    if (ef_s <= 64) { *pool_slots = 64; return frog_search_kernel<2, MODE, BITMAP, F16>; }
+    if (ef_s <= 128) { *pool_slots = 128; return frog_search_kernel<4, MODE, BITMAP, F16>; }
+    if (ef_s <= 256) { *pool_slots = 256; return frog_search_kernel<8, MODE, BITMAP, F16>; }
     *pool_slots = 512;
-    return frog_search_kernel<16, MODE, BITMAP>;
+    return frog_search_kernel<16, MODE, BITMAP, F16>;
 }
 
 struct LaunchPlan {
@@ -464,15 +467,21 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
                 LaunchPlan* out) {
     int pool_slots = 0;
     kernel_fn fn;
-    if (bitmap)
-        fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, true>(beam_width, &pool_slots)
-           : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, true>(beam_width, &pool_slots)
-                                  : pick_kernel<MODE_FAST, true>(beam_width, &pool_slots);
+    const bool f16 = P.storage == FROG_STORAGE_F16;
+    if (f16 && !bitmap) return FROG_ERR_UNSUPPORTED;       // fp16 rows are read by the bitmap kernels only
+    if (f16)
+        fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, true, true>(beam_width, &pool_slots)
+           : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, true, true>(beam_width, &pool_slots)
+                                  : pick_kernel<MODE_FAST, true, true>(beam_width, &pool_slots);
+    else if (bitmap)
+        fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, true, false>(beam_width, &pool_slots)
+           : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, true, false>(beam_width, &pool_slots)
+                                  : pick_kernel<MODE_FAST, true, false>(beam_width, &pool_slots);
     else
-        fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, false>(beam_width, &pool_slots)
-           : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, false>(beam_width, &pool_slots)
-                                  : pick_kernel<MODE_FAST, false>(beam_width, &pool_slots);
-    size_t smem = warp_smem_bytes(pool_slots, ix->info.d_pad, P.hash_bits, bitmap) * WARPS_PER_CTA;
+        fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, false, false>(beam_width, &pool_slots)
+           : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, false, false>(beam_width, &pool_slots)
+                                  : pick_kernel<MODE_FAST, false, false>(beam_width, &pool_slots);
+    size_t smem = warp_smem_bytes(pool_slots, query_len(ix->info.d), P.hash_bits, bitmap) * WARPS_PER_CTA;
     if (smem > 227 * 1024) return FROG_ERR_UNSUPPORTED;
     FROG_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
@@ -489,6 +498,21 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
     out->ctas_per_sm = per_sm;
     out->smem = smem;
     return FROG_OK;
+}
+
+// gather source and stage geometry: a row slot is the row (or its 512-byte chunk) rounded up to a
+// power of two; as many rows as fit the stage buffer (at most 16, a multiple of 4) share one phase
+void set_gather(const frog_index* ix, bool f16, FrogSearchArgs* A) {
+    const int d_pad_h = query_len(ix->info.d);
+    A->rows = f16 ? ix->d_vectors_h : (const void*)ix->d_vectors;
+    A->row_bytes = f16 ? d_pad_h * 2 : ix->info.d_pad * 4;
+    int slot = 16;
+    while (slot < A->row_bytes && slot < STAGE_CHUNK) slot <<= 1;
+    A->slot_bytes = slot;
+    int rows = STAGE_BYTES / slot;
+    rows = rows > 16 ? 16 : rows;
+    A->rows_per_pass = rows < 4 ? 4 : rows / 4 * 4;
+    A->q_len = d_pad_h;
 }
 
 // per-warp visited slab: one bit per rank, padded to 128 bytes
@@ -520,6 +544,8 @@ int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in
     if (P.hash_bits < 6 || P.hash_bits > 15) return FROG_ERR_INVALID_ARG;
     if (P.visited != FROG_VISITED_AUTO && P.visited != FROG_VISITED_BITMAP && P.visited != FROG_VISITED_HASH)
         return FROG_ERR_INVALID_ARG;
+    if (P.storage != FROG_STORAGE_F32 && P.storage != FROG_STORAGE_F16) return FROG_ERR_INVALID_ARG;
+    if (P.storage == FROG_STORAGE_F16 && !ix->d_vectors_h) return FROG_ERR_INVALID_ARG;   // not enabled on this index
     (void)ix;
     *out = P;
     return FROG_OK;
@@ -643,6 +669,7 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     A.bitmap_words = bitmap_words_per_slot(index);
     A.ranges = nullptr;
     A.order = nullptr;
+    set_gather(index, P.storage == FROG_STORAGE_F16, &A);
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     FROG_CUDA_TRY(cudaMemsetAsync(index->d_work, 0, 1024, s));
@@ -768,6 +795,7 @@ extern "C" int frog_search_static(const frog_index_t* index, const float* querie
     A.bitmap_words = words;
     A.ranges = nullptr;                                     // endpoints and order are computed in the kernel
     A.order = nullptr;
+    set_gather(index, P.storage == FROG_STORAGE_F16, &A);
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the array keeps what the previous call left: the counter must restart at zero; every warp
@@ -778,3 +806,37 @@ extern "C" int frog_search_static(const frog_index_t* index, const float* querie
     return FROG_OK;
 }
 
+
+// ---- optional fp16 copy of the vectors (paper Sec. 8.1.4: its GPU programs compute distances from
+// float16 data with float32 accumulation) ---------------------------------------------------------
+namespace {
+__global__ void to_half_kernel(const float* __restrict__ src, int d_pad, __half* __restrict__ dst, int d_pad_h, size_t n) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n * (size_t)d_pad_h) return;
+    const size_t r = i / d_pad_h;
+    const int c = (int)(i - r * d_pad_h);
+    dst[i] = __float2half_rn(c < d_pad ? src[r * d_pad + c] : 0.f);
+}
+}  // namespace
+
+extern "C" int frog_index_enable_f16(frog_index_t* ix) {
+    if (!ix) return FROG_ERR_INVALID_ARG;
+    if (ix->d_vectors_h) return FROG_OK;
+    FROG_CUDA_TRY(cudaSetDevice(ix->info.device));
+    const int d_pad_h = query_len(ix->info.d);
+    const size_t elems = (size_t)ix->info.n * d_pad_h;
+    cudaError_t e = cudaMalloc(&ix->d_vectors_h, elems * sizeof(__half));
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        froghost::set_cuda_error(e);
+        ix->d_vectors_h = nullptr;
+        return FROG_ERR_NOMEM;
+    }
+    to_half_kernel<<<(unsigned)((elems + 255) / 256), 256>>>(ix->d_vectors, ix->info.d_pad,
+                                                             static_cast<__half*>(ix->d_vectors_h), d_pad_h,
+                                                             (size_t)ix->info.n);
+    FROG_CUDA_TRY(cudaGetLastError());
+    FROG_CUDA_TRY(cudaDeviceSynchronize());
+    ix->info.device_bytes += (int64_t)(elems * sizeof(__half));
+    return FROG_OK;
+}

@@ -252,3 +252,40 @@ def test_index_info_and_from_host(libs, tiny):
     _assert_parity(got, ref)
     g2.close()
     gix.close()
+
+
+# ---- half-precision storage -----------------------------------------------------------------------
+@pytest.mark.parametrize("name,n,nq", [("tiny", 10_000, 200), ("deep1m", 50_000, 300), ("text", 20_000, 100),
+                                        ("sift", 60_000, 300)])
+def test_f16_storage_equals_oracle_on_rounded_vectors(libs, cache_dir, name, n, nq):
+    """fp16 storage, fp32 arithmetic: bit-exact against the oracle run on the fp16-rounded vectors;
+    recall against the fp32 ground truth stays close to the fp32 search."""
+    from conftest import build_scaled
+    wl, path, ix = build_scaled(libs, cache_dir, name, n, nq)
+    ix16 = oracle.rounded_to_f16(ix)
+    gix = libs.Index.load(path, 0)
+    try:
+        gix.enable_f16()
+        gix.enable_f16()                                    # idempotent
+        for ef, B in ((48, 16), (64, 32)):
+            ref = oracle.search(ix16, wl.queries, wl.lo, wl.hi, 10, ef, B=B, trace_cap=60000)
+            got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, 10, ef, trace_cap=60000, budget=B,
+                              storage=libs.STORAGE_F16)
+            _assert_parity(got, ref, slots=_default_slots(ef))
+            assert np.array_equal(got[3], ref.stats)
+        gt, _, _ = oracle.exact_slab(ix, wl.queries, wl.lo, wl.hi, 10, mode=0)
+        ref32 = oracle.search(ix, wl.queries, wl.lo, wl.hi, 10, 64, B=32)
+        assert abs(oracle.recall(got[0], gt) - oracle.recall(ref32.ids, gt)) <= 0.01
+        if name == "sift":
+            # integer components 0..255 are exact in fp16: the two storages give the same answer
+            assert np.array_equal(got[0], ref32.ids) and np.array_equal(got[1], ref32.dists)
+        # the request is refused where it cannot be served
+        with pytest.raises(libs.FrogError):
+            _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, 10, 32, storage=libs.STORAGE_F16,
+                        visited=libs.VISITED_HASH)
+    finally:
+        gix.close()
+    g2 = libs.Index.load(path, 0)
+    with pytest.raises(libs.FrogError):                      # not enabled on this handle
+        _gpu_search(libs, g2, wl.queries, wl.lo, wl.hi, 10, 32, storage=libs.STORAGE_F16)
+    g2.close()
