@@ -315,10 +315,17 @@ __device__ __forceinline__ float staged_dist2(const float* __restrict__ vectors,
 // `rows_per_pass` (<= 16, multiple of 4) rows complete on one mbarrier phase.  fp16 elements are
 // converted to fp32 on the way out of shared memory; products and sums are fp32 in the same fixed
 // order, so the result equals the fp32 routine run on the rounded values bit for bit.
-template <bool F16>
+// ROWB > 0 fixes the row size (and with it slot size and rows per pass) at compile time, which
+// unrolls the inner loops for the common shapes; ROWB == 0 takes the geometry from the arguments.
+template <bool F16, int ROWB = 0>
 __device__ __forceinline__ float staged_dist2_flex(const void* __restrict__ rows, int row_bytes, int slot_bytes,
                                                    int rows_per_pass, const float4* qs, float4* stage, uint64_t* bar,
                                                    uint32_t& phase, bool& ok, uint32_t my_rank, int ns, int lane) {
+    if (ROWB > 0) {
+        row_bytes = ROWB;
+        slot_bytes = ROWB >= STAGE_CHUNK ? STAGE_CHUNK : ROWB;     // ROWB is a power of two when below 512
+        rows_per_pass = (8 * STAGE_CHUNK / slot_bytes) > 16 ? 16 : (8 * STAGE_CHUNK / slot_bytes);
+    }
     const int team = lane >> 3, sub = lane & 7;
     constexpr int GROUP_BYTES = F16 ? 8 : 16;             // 4 elements
     float out = 0.f;

@@ -95,7 +95,7 @@ __device__ __forceinline__ bool visited_test_and_set(const WarpSmem& S, uint32_t
 // Distances of the ns <= 32 ranks listed in cand[0..ns) and their merge into the pool (Alg. 2
 // lines 14-17).  Returns the first unexpanded pool position.  Kept out of line: it is called from
 // three places of the kernel and inlining every copy costs registers and instruction cache.
-template <int EPL, bool F16>
+template <int EPL, bool F16, int ROWB>
 __device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows, int row_bytes, int slot_bytes,
                                                    int rows_per_pass, int ef_s,
                                                    uint64_t* pool, const uint32_t* cand, uint64_t* bar,
@@ -125,7 +125,7 @@ __device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows
         __syncwarp();                       // lane 0's update of the parity in the previous call
         uint32_t phase = bar_words[0];
         bool ok = true;
-        d2 = staged_dist2_flex<F16>(rows, row_bytes, slot_bytes, rows_per_pass, qs, stage, bar, phase, ok, id, ns, lane);
+        d2 = staged_dist2_flex<F16, ROWB>(rows, row_bytes, slot_bytes, rows_per_pass, qs, stage, bar, phase, ok, id, ns, lane);
         __syncwarp();                       // every lane has read the old parity
         if (lane == 0) {
             bar_words[0] = phase;
@@ -154,7 +154,7 @@ __device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows
     return (int)merge_batch<EPL>(pool, key, ef_s, lane);
 }
 
-template <int EPL, int MODE, bool BITMAP, bool F16>
+template <int EPL, int MODE, bool BITMAP, bool F16, int ROWB = 0>
 __global__ void __launch_bounds__(WARPS_PER_CTA * 32, MODE == MODE_FAST ? (EPL <= 4 ? FROG_MINB : 4) : 1)
 frog_search_kernel(const FrogSearchArgs A) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -206,7 +206,7 @@ frog_search_kernel(const FrogSearchArgs A) {
         int enc_hot_bytes = 0;                    // bytes of the first two chunks of a vertex's hotspot
         int second_pos = NO_POS;                  // pool position of the next unexpanded entry after `first`
         auto EVAL = [&](int ns_, uint32_t flag_) {
-            int f_ = evaluate_and_merge<EPL, F16>(A.rows, A.row_bytes, A.slot_bytes, A.rows_per_pass, A.ef_s, S.pool,
+            int f_ = evaluate_and_merge<EPL, F16, ROWB>(A.rows, A.row_bytes, A.slot_bytes, A.rows_per_pass, A.ef_s, S.pool,
                                                   S.cand, S.bar, S.q, S.stage, ns_, flag_, !BITMAP, enc_hot_base,
                                                   (size_t)A.H * A.m, enc_hot_bytes, second_pos,
                                                   MODE == MODE_PROFILE ? &t_split : nullptr);
@@ -481,6 +481,14 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
         fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, false, false>(beam_width, &pool_slots)
            : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, false, false>(beam_width, &pool_slots)
                                   : pick_kernel<MODE_FAST, false, false>(beam_width, &pool_slots);
+    // common shape with the geometry fixed at compile time: fp32 rows of 512 bytes (d = 125..128)
+    if (mode == MODE_FAST && bitmap && !f16 && ix->info.d_pad == 128) {
+        if (beam_width <= 32) fn = frog_search_kernel<1, MODE_FAST, true, false, 512>;
+        else if (beam_width <= 64) fn = frog_search_kernel<2, MODE_FAST, true, false, 512>;
+        else if (beam_width <= 128) fn = frog_search_kernel<4, MODE_FAST, true, false, 512>;
+        else if (beam_width <= 256) fn = frog_search_kernel<8, MODE_FAST, true, false, 512>;
+        else fn = frog_search_kernel<16, MODE_FAST, true, false, 512>;
+    }
     size_t smem = warp_smem_bytes(pool_slots, query_len(ix->info.d), P.hash_bits, bitmap) * WARPS_PER_CTA;
     if (smem > 227 * 1024) return FROG_ERR_UNSUPPORTED;
     FROG_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
