@@ -41,7 +41,8 @@ enum {
 
 /* Limits of the search kernels. */
 #define FROG_MAX_BEAM_WIDTH 512 /* ef_s */
-#define FROG_MAX_BUDGET 32      /* B and epn */
+#define FROG_MAX_BUDGET 64      /* expansion budget B */
+#define FROG_MAX_EPN 32         /* entry points */
 
 typedef struct {
     int64_t n;          /* objects */
@@ -61,7 +62,7 @@ typedef struct {
 /* Optional query-time parameters (Alg. 2 arguments other than k and ef_s). */
 typedef struct {
     int32_t epn;        /* entry points, 1..32; 0 = default 16 (paper Sec. 8.1.4) */
-    int32_t budget;     /* expansion budget B, 1..32; 0 = default 16 */
+    int32_t budget;     /* expansion budget B, 1..64; 0 = default 16 */
     int32_t max_iters;  /* hard cap on expansions per query; 0 = default 16 * beam_width */
     int32_t no_hotspot; /* nonzero: scan all H layers instead of the hotspot (ablation) */
     uint64_t seed;      /* seed of the entry-point generator */

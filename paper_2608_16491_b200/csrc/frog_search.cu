@@ -62,7 +62,7 @@ struct WarpSmem {
 };
 
 inline size_t warp_smem_bytes(int pool_slots, int q_len, int hash_bits, bool bitmap) {
-    return (size_t)pool_slots * 8 + 32 * 4 + 16 + (size_t)q_len * 4 + STAGE_BYTES +
+    return (size_t)pool_slots * 8 + 64 * 4 + 16 + (size_t)q_len * 4 + STAGE_BYTES +
            (bitmap ? 0 : ((size_t)4 << hash_bits));
 }
 inline int query_len(int d) { return (d + 7) / 8 * 8; }
@@ -162,12 +162,12 @@ frog_search_kernel(const FrogSearchArgs A) {
     const int warp = threadIdx.x >> 5;
     constexpr int POOL = 32 * EPL;
     const int hash_slots = BITMAP ? 0 : (1 << A.hash_bits);
-    const size_t per_warp = (size_t)POOL * 8 + 32 * 4 + 16 + (size_t)A.q_len * 4 + STAGE_BYTES + (size_t)hash_slots * 4;
+    const size_t per_warp = (size_t)POOL * 8 + 64 * 4 + 16 + (size_t)A.q_len * 4 + STAGE_BYTES + (size_t)hash_slots * 4;
     unsigned char* base = smem_raw + per_warp * warp;
     WarpSmem S;
     S.pool = reinterpret_cast<uint64_t*>(base);
     S.cand = reinterpret_cast<uint32_t*>(S.pool + POOL);
-    S.bar = reinterpret_cast<uint64_t*>(S.cand + 32);
+    S.bar = reinterpret_cast<uint64_t*>(S.cand + 64);
     S.q = reinterpret_cast<float4*>(S.bar + 2);
     S.stage = reinterpret_cast<float4*>(reinterpret_cast<float*>(S.q) + A.q_len);
     S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(S.stage) + STAGE_BYTES);
@@ -205,9 +205,9 @@ frog_search_kernel(const FrogSearchArgs A) {
         const uint32_t* enc_hot_base = nullptr;   // ENC rows from L_start on (set once the hotspot is known)
         int enc_hot_bytes = 0;                    // bytes of the first two chunks of a vertex's hotspot
         int second_pos = NO_POS;                  // pool position of the next unexpanded entry after `first`
-        auto EVAL = [&](int ns_, uint32_t flag_) {
+        auto EVAL = [&](int ns_, uint32_t flag_, int off_ = 0) {
             int f_ = evaluate_and_merge<EPL, F16, ROWB>(A.rows, A.row_bytes, A.slot_bytes, A.rows_per_pass, A.ef_s, S.pool,
-                                                  S.cand, S.bar, S.q, S.stage, ns_, flag_, !BITMAP, enc_hot_base,
+                                                  S.cand + off_, S.bar, S.q, S.stage, ns_, flag_, !BITMAP, enc_hot_base,
                                                   (size_t)A.H * A.m, enc_hot_bytes, second_pos,
                                                   MODE == MODE_PROFILE ? &t_split : nullptr);
             if (MODE == MODE_PROFILE) {
@@ -364,7 +364,13 @@ frog_search_kernel(const FrogSearchArgs A) {
                         trace_ok = false;
                     }
                 }
-                packed = EVAL(ns, 0u);   // lines 14-17
+                // lines 14-17; a budget above 32 can leave up to 64 survivors: two batches, the pool
+                // after both is the same as after one merge of all of them
+                packed = EVAL(min(ns, 32), 0u);
+                if (ns > 32) {
+                    second_pos = (packed >> 16) & 0xFFFF;
+                    packed = EVAL(ns - 32, 0u, 32);
+                }
                 first = packed & 0xFFFF;
                 second_pos = (packed >> 16) & 0xFFFF;
             }
@@ -540,7 +546,7 @@ int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in
     if (P.epn == 0) P.epn = 16;
     if (P.budget == 0) P.budget = 16;
     if (P.max_iters == 0) P.max_iters = 16 * beam_width;
-    if (P.epn < 1 || P.epn > FROG_MAX_BUDGET || P.budget < 1 || P.budget > FROG_MAX_BUDGET || P.max_iters < 1)
+    if (P.epn < 1 || P.epn > FROG_MAX_EPN || P.budget < 1 || P.budget > FROG_MAX_BUDGET || P.max_iters < 1)
         return FROG_ERR_INVALID_ARG;
     if (P.hash_bits == 0) {
         // about 16 evaluated vertices per beam slot, at most half full

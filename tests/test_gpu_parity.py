@@ -94,11 +94,13 @@ def test_tiny_plain_call_equals_ex_call(libs, tiny_gpu):
     assert np.array_equal(dists.cpu().numpy(), ref.dists)
 
 
-@pytest.mark.parametrize("params", [dict(epn=1), dict(epn=32), dict(budget=4), dict(budget=32),
+@pytest.mark.parametrize("params", [dict(epn=1), dict(epn=32), dict(budget=4), dict(budget=32), dict(budget=48),
+                                    dict(budget=64), dict(budget=64, visited=2), dict(budget=40, no_hotspot=1),
                                     dict(no_hotspot=1), dict(seed=12345), dict(max_iters=7),
                                     dict(epn=7, budget=9, seed=3)])
 def test_tiny_parameter_variants(libs, tiny_gpu, params):
     wl, ix, gix = tiny_gpu
+    params = dict(params)
     okw = dict(epn=params.get("epn", 16), B=params.get("budget", 16), seed=params.get("seed", 0),
                no_hotspot=bool(params.get("no_hotspot", 0)), max_iters=params.get("max_iters", 0))
     ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 48, trace_cap=20000, **okw)
@@ -150,6 +152,8 @@ def test_empty_batch_and_argument_errors(libs, tiny_gpu):
         assert e.value.code == 1
     with pytest.raises(libs.FrogError):
         gix.search(q, lo, hi, 10, 32, params=libs.Params(epn=33))
+    with pytest.raises(libs.FrogError):
+        gix.search(q, lo, hi, 10, 32, params=libs.Params(budget=65))
     # a failed call leaves the index usable
     ids, _ = gix.search(q, lo, hi, 10, 32)
     torch.cuda.synchronize()
@@ -204,7 +208,8 @@ def test_scaled_workloads_match_oracle(libs, cache_dir, name, n, nq):
     gix = libs.Index.load(path, 0)
     try:
         for ef, k, B, vis in ((32, 10, 16, libs.VISITED_BITMAP), (100, 100, 16, libs.VISITED_HASH),
-                              (64, 10, 32, libs.VISITED_BITMAP), (48, 10, 24, libs.VISITED_HASH)):
+                              (64, 10, 32, libs.VISITED_BITMAP), (48, 10, 24, libs.VISITED_HASH),
+                              (48, 10, 64, libs.VISITED_BITMAP)):
             ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef, B=B, trace_cap=60000)
             got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, k, ef, trace_cap=60000, budget=B, visited=vis)
             _assert_parity(got, ref, slots=_default_slots(ef))
