@@ -245,6 +245,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t phase) {
 // 4-float groups g = s, s+8, ... in increasing g, fused multiply-adds, butterfly 4-2-1), so both
 // routines return identical bits.  `phase` is the running parity of the warp's mbarrier.
 constexpr int STAGE_CHUNK = 512;     // bytes of one row in flight per pass
+#ifndef FROG_STAGE_ROWS
+#define FROG_STAGE_ROWS 8            // 512-byte row slots in the search kernel's stage buffer
+#endif
 template <int STAGE_ROWS>
 __device__ __forceinline__ float staged_dist2(const float* __restrict__ vectors, int d_pad, const float4* qs,
                                               float4* stage, uint64_t* bar, uint32_t& phase, bool& ok,
@@ -324,15 +327,15 @@ __device__ __forceinline__ float staged_dist2_flex(const void* __restrict__ rows
     if (ROWB > 0) {
         row_bytes = ROWB;
         slot_bytes = ROWB >= STAGE_CHUNK ? STAGE_CHUNK : ROWB;     // ROWB is a power of two when below 512
-        rows_per_pass = (8 * STAGE_CHUNK / slot_bytes) > 16 ? 16 : (8 * STAGE_CHUNK / slot_bytes);
+        rows_per_pass = (FROG_STAGE_ROWS * STAGE_CHUNK / slot_bytes) > 16 ? 16 : (FROG_STAGE_ROWS * STAGE_CHUNK / slot_bytes);
     }
     const int team = lane >> 3, sub = lane & 7;
     constexpr int GROUP_BYTES = F16 ? 8 : 16;             // 4 elements
     float out = 0.f;
-    const int src = (lane & 3) << 3;
 #pragma unroll 1
     for (int r0 = 0; r0 < ns; r0 += rows_per_pass) {
         const int nrows = min(rows_per_pass, ns - r0);
+        const int src = ((lane - r0) & 3) << 3;             // team that summed this lane's row
         const uint32_t copy_rank = __shfl_sync(FULL, my_rank, (r0 + lane) & 31);
         const char* src_row = reinterpret_cast<const char*>(rows) + (size_t)copy_rank * (size_t)row_bytes;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};

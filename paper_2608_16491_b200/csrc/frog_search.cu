@@ -24,7 +24,10 @@ using namespace frogdev;
 
 namespace {
 
-constexpr int WARPS_PER_CTA = 2;
+#ifndef FROG_WARPS_PER_CTA
+#define FROG_WARPS_PER_CTA 2
+#endif
+constexpr int WARPS_PER_CTA = FROG_WARPS_PER_CTA;
 #ifndef FROG_MINB
 #define FROG_MINB 16          // resident CTAs per SM the register allocation aims at (EPL <= 4)
 #endif
@@ -32,6 +35,9 @@ constexpr int WARPS_PER_CTA = 2;
 #define FROG_NG 2
 #endif
 
+#ifndef FROG_MINB_BIG
+#define FROG_MINB_BIG 4       // the same for pools above 128 entries
+#endif
 #ifndef FROG_EVAL_INLINE
 #define FROG_EVAL_INLINE __noinline__
 #endif
@@ -45,9 +51,6 @@ constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2;
 #endif
 #ifndef FROG_ENC_LD
 #define FROG_ENC_LD ldg_stream_u32
-#endif
-#ifndef FROG_STAGE_ROWS
-#define FROG_STAGE_ROWS 8     // rows the copy engine stages per pass (8 or 16), 512 bytes each
 #endif
 constexpr int STAGE_BYTES = FROG_STAGE_ROWS * STAGE_CHUNK;
 
@@ -155,7 +158,7 @@ __device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows
 }
 
 template <int EPL, int MODE, bool BITMAP, bool F16, int ROWB = 0>
-__global__ void __launch_bounds__(WARPS_PER_CTA * 32, MODE == MODE_FAST ? (EPL <= 4 ? FROG_MINB : 4) : 1)
+__global__ void __launch_bounds__(WARPS_PER_CTA * 32, MODE == MODE_FAST ? (EPL <= 4 ? FROG_MINB : FROG_MINB_BIG) : 1)
 frog_search_kernel(const FrogSearchArgs A) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int lane = lane_id();
@@ -501,6 +504,9 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
     int per_sm = 0;
     FROG_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)fn, WARPS_PER_CTA * 32, smem));
     if (per_sm < 1) return FROG_ERR_UNSUPPORTED;
+#ifdef FROG_CAP_CTAS
+    if (per_sm > FROG_CAP_CTAS) per_sm = FROG_CAP_CTAS;
+#endif
     int grid = per_sm * ix->sm_count;
     if (nq > 0) {
         int need = (nq + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
@@ -525,7 +531,7 @@ void set_gather(const frog_index* ix, bool f16, FrogSearchArgs* A) {
     A->slot_bytes = slot;
     int rows = STAGE_BYTES / slot;
     rows = rows > 16 ? 16 : rows;
-    A->rows_per_pass = rows < 4 ? 4 : rows / 4 * 4;
+    A->rows_per_pass = rows;
     A->q_len = d_pad_h;
 }
 
