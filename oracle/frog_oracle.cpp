@@ -240,6 +240,7 @@ struct Params {
     uint64_t seed;
     int warp;        // chunk width of Alg. 4 (32; any value gives the same EN list)
     int no_hotspot;  // ablation: scan all H layers
+    int exact_below; // ranges of at most this many objects are answered by the exact scan too (0: off)
 };
 
 // status bits
@@ -263,14 +264,16 @@ void search_one(const Index& ix, const float* v_q, int32_t lo, int32_t hi, int k
     std::vector<Cand> pool;
     if (lo > hi || w <= 0) {
         st |= ST_EMPTY;
-    } else if (w <= ef_s) {
-        // every valid object enters the pool: the answer is exact
+    } else if (w <= ef_s || w <= P.exact_below) {
+        // every valid object is evaluated and the pool keeps the ef_s nearest: the answer is exact
+        // (Def. 2 over the contiguous rank slab of Sec. 4)
         st |= ST_EXACT;
         for (int64_t r = l_q; r <= r_q; ++r) {
             pool.push_back(Cand{dist2_canonical(v_q, ix.vectors + r * ix.d_pad, ix.d_pad), (uint32_t)r, 1});
             ++n_dist;
         }
         std::sort(pool.begin(), pool.end(), cand_less);
+        if ((int)pool.size() > ef_s) pool.resize(ef_s);
     } else {
         int L_start, L_end;
         hotspot_localization(l_q, r_q, ix.H, ix.n, &L_start, &L_end);        // line 1
@@ -365,11 +368,11 @@ int frog_oracle_search(const int32_t* sorted_attr, const int32_t* rank2id, const
                        const uint32_t* enc, int64_t n, int d_pad, int H, int m,
                        const float* queries, const int32_t* lo, const int32_t* hi, int64_t nq,
                        int k, int ef_s, int epn, int B, int max_iters, uint64_t seed, int warp,
-                       int no_hotspot,
+                       int no_hotspot, int exact_below,
                        int32_t* out_ids, float* out_dists, uint32_t* status, uint32_t* stats,
                        uint32_t* trace_out, int64_t trace_cap, int threads) {
     Index ix{sorted_attr, rank2id, vectors, enc, n, d_pad, H, m};
-    Params P{epn, B, max_iters, seed, warp, no_hotspot};
+    Params P{epn, B, max_iters, seed, warp, no_hotspot, exact_below};
     int used = 1;
 #ifdef _OPENMP
     omp_set_num_threads(threads > 0 ? threads : omp_get_num_procs());   // <= 0: all cores

@@ -208,9 +208,10 @@ frog_search_kernel(const FrogSearchArgs A) {
         const uint32_t* enc_hot_base = nullptr;   // ENC rows from L_start on (set once the hotspot is known)
         int enc_hot_bytes = 0;                    // bytes of the first two chunks of a vertex's hotspot
         int second_pos = NO_POS;                  // pool position of the next unexpanded entry after `first`
-        auto EVAL = [&](int ns_, uint32_t flag_, int off_ = 0) {
+        auto EVAL = [&](int ns_, uint32_t flag_, int off_ = 0, bool last_ = true) {
             int f_ = evaluate_and_merge<EPL, F16, ROWB>(A.rows, A.row_bytes, A.slot_bytes, A.rows_per_pass, A.ef_s, S.pool,
-                                                  S.cand + off_, S.bar, S.q, S.stage, ns_, flag_, !BITMAP, enc_hot_base,
+                                                  S.cand + off_, S.bar, S.q, S.stage, ns_, flag_, !BITMAP,
+                                                  last_ ? enc_hot_base : nullptr,
                                                   (size_t)A.H * A.m, enc_hot_bytes, second_pos,
                                                   MODE == MODE_PROFILE ? &t_split : nullptr);
             if (MODE == MODE_PROFILE) {
@@ -369,10 +370,11 @@ frog_search_kernel(const FrogSearchArgs A) {
                 }
                 // lines 14-17; a budget above 32 can leave up to 64 survivors: two batches, the pool
                 // after both is the same as after one merge of all of them
-                packed = EVAL(min(ns, 32), 0u);
                 if (ns > 32) {
-                    second_pos = (packed >> 16) & 0xFFFF;
+                    second_pos = EVAL(32, 0u, 0, false) & 0xFFFF;   // the next unexpanded entry so far
                     packed = EVAL(ns - 32, 0u, 32);
+                } else {
+                    packed = EVAL(ns, 0u);
                 }
                 first = packed & 0xFFFF;
                 second_pos = (packed >> 16) & 0xFFFF;

@@ -293,6 +293,27 @@ def test_small_ranges_are_exact_and_padded(tiny_runs):
     assert seen_exact > 0
 
 
+def test_exact_below_extends_the_exact_rule(tiny_runs):
+    """With exact_below = T every range of at most max(ef_s, T) objects equals the definition
+    scan (ids and distances), the others are searched as before."""
+    wl, ix, gt_ids, gt_d, runs = tiny_runs
+    ef, T = 16, 700
+    res = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, ef, exact_below=T)
+    base = runs[ef]
+    n_ext = 0
+    for q in range(wl.nq):
+        l, r = oracle.rank_interval(ix.sorted_attr, int(wl.lo[q]), int(wl.hi[q]))
+        w = r - l + 1
+        if 0 < w <= T:
+            n_ext += w > ef
+            assert res.status[q] & oracle.ST_EXACT
+            assert np.array_equal(res.ids[q], gt_ids[q]) and np.array_equal(res.dists[q], gt_d[q])
+            assert res.stats[q, 3] == w and res.stats[q, 0] == 0
+        else:
+            assert np.array_equal(res.ids[q], base.ids[q]) and np.array_equal(res.stats[q], base.stats[q])
+    assert n_ext > 10
+
+
 def test_range_with_at_most_k_points_returns_exactly_those(tiny):
     wl, _, ix = tiny
     srt = np.asarray(ix.sorted_attr)
