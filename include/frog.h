@@ -71,6 +71,11 @@ typedef struct {
     int32_t storage;    /* FROG_STORAGE_*: which copy of the vectors the gather reads */
     int32_t debug_flags;/* bit 0: with `trace`, record per-phase cycle counts instead of EN lists;
                            bit 1: process queries in input order (no heaviest-first planning pass) */
+    int32_t exact_below;/* ranges holding at most max(beam_width, exact_below) objects are answered by
+                           scanning their contiguous rank slab (exact, status FROG_ST_EXACT) instead of
+                           the graph search; 0 = default: only ranges that fit the pool.  Not in the
+                           paper, whose smallest ranges hold thousands of objects (Sec. 8.1.2) */
+    int32_t reserved;   /* must be 0 */
 } frog_params_t;
 
 /* Vector storage read by the search.  F32 (default): the index's fp32 rows.  F16: an fp16 copy made
@@ -90,7 +95,7 @@ typedef struct {
 
 /* Per-query status bits written by frog_search_ex. */
 #define FROG_ST_EMPTY 1u     /* lo > hi or no object in [lo, hi]: row is all padding */
-#define FROG_ST_EXACT 2u     /* range holds <= beam_width objects: answered by exact scan */
+#define FROG_ST_EXACT 2u     /* range holds <= max(beam_width, exact_below) objects: answered by exact scan */
 #define FROG_ST_ITER_CAP 4u  /* expansion cap hit; the current pool was returned */
 #define FROG_ST_SHORT 8u     /* fewer than k results; tail is padding */
 #define FROG_ST_COPY_TIMEOUT 32u /* a bulk copy into shared memory did not complete within the kernel's

@@ -182,9 +182,10 @@ def default_max_iters(ef_s: int) -> int:
 def search(ix: OracleIndex, queries: np.ndarray, lo: np.ndarray, hi: np.ndarray, k: int, ef_s: int,
            epn: int = 16, B: int = 16, max_iters: int = 0, seed: int = 0, warp: int = 32,
            no_hotspot: bool = False, trace_cap: int = 0, threads: int = 0,
-           exact_below: int = 0) -> SearchResult:
+           exact_below: int = 0, eager_hash: bool = False) -> SearchResult:
     """Alg. 2 over the whole batch (parallel over queries only).  Ranges holding at most
-    max(ef_s, exact_below) objects are answered by the exact slab scan."""
+    max(ef_s, exact_below) objects are answered by the exact slab scan.  eager_hash: ablation with
+    the visited test inside the predicate of Alg. 4."""
     q = pad_queries(queries, ix.d_pad)
     nq = q.shape[0]
     lo = np.ascontiguousarray(lo, dtype=np.int32)
@@ -201,7 +202,7 @@ def search(ix: OracleIndex, queries: np.ndarray, lo: np.ndarray, hi: np.ndarray,
         _p(ix.enc, C.c_uint32), C.c_int64(ix.n), C.c_int(ix.d_pad), C.c_int(ix.H), C.c_int(ix.m),
         _p(q, C.c_float), _p(lo, C.c_int32), _p(hi, C.c_int32), C.c_int64(nq),
         C.c_int(k), C.c_int(ef_s), C.c_int(epn), C.c_int(B), C.c_int(max_iters), C.c_uint64(seed),
-        C.c_int(warp), C.c_int(1 if no_hotspot else 0), C.c_int(exact_below),
+        C.c_int(warp), C.c_int(1 if no_hotspot else 0), C.c_int(exact_below), C.c_int(1 if eager_hash else 0),
         _p(ids, C.c_int32), _p(dists, C.c_float), _p(status, C.c_uint32), _p(stats, C.c_uint32),
         _p(trace, C.c_uint32), C.c_int64(trace_cap), C.c_int(threads))
     return SearchResult(ids, dists, status, stats, trace, int(used))

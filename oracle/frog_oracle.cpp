@@ -23,7 +23,10 @@
 //     ties are decided on the squared value, ties broken by rank; reported distance =
 //     sqrtf(squared).
 //   * visited set: exact, never erased.  Hard cap on expansions (max_iters).
-//   * a range holding at most ef_s objects is answered exactly (every object enters the pool).
+//   * a range holding at most ef_s objects is answered exactly (every object enters the pool);
+//     the option exact_below = T extends this to ranges of at most max(ef_s, T) objects.
+//   * ablation options: no_hotspot (scan all H layers), eager_hash (visited test inside the
+//     predicate of Alg. 4 instead of after selection and budget).
 //
 // Parity unpinned by the paper: the +-1 convention of Eq. 6 (pinned only by the reading
 // above), and recall levels (the paper's curves are figures on datasets not available here).
@@ -155,6 +158,43 @@ int en_identification(const uint32_t* enc_u, int m, int64_t l_q, int64_t r_q,
 }
 
 // ---------------------------------------------------------------------------------------------
+// Ablation of the lazy hash check (Sec. 6.2): the EAGER form puts the visited test into the
+// predicate of Alg. 4, so an id that was already evaluated neither occupies a slot nor consumes
+// budget.  Chunk semantics as in Alg. 4: all lanes of a chunk test against the visited set as it
+// stood when the chunk was loaded; the admitted prefix is then inserted, in order (a second copy
+// of an id inside the same chunk is admitted, fails the insertion and is not evaluated).
+// `fresh` receives the admitted ids that were inserted, in order.
+// ---------------------------------------------------------------------------------------------
+int en_identification_eager(const uint32_t* enc_u, int m, int64_t l_q, int64_t r_q,
+                            int L_start, int L_end, int B, int warp, std::set<uint32_t>& visited,
+                            uint32_t* EN, std::vector<uint32_t>& fresh, int* rows_read) {
+    int size_EN = 0;
+    int rows = 0;
+    fresh.clear();
+    if (B <= 0) { if (rows_read) *rows_read = 0; return 0; }
+    const uint32_t* hot = enc_u + (int64_t)L_start * m;
+    int total = (L_end - L_start + 1) * m;
+    for (int c0 = 0; c0 < total; c0 += warp) {
+        int c1 = std::min(total, c0 + warp);
+        rows = (c1 + m - 1) / m;
+        std::vector<uint32_t> pass;
+        for (int lane = 0; lane < c1 - c0; ++lane) {
+            uint32_t v = hot[c0 + lane];
+            bool pred = (v != BOT) && (l_q <= (int64_t)v) && ((int64_t)v <= r_q) && !visited.count(v);
+            if (pred) pass.push_back(v);
+        }
+        int a = std::min<int>((int)pass.size(), B - size_EN);
+        for (int j = 0; j < a; ++j) {
+            EN[size_EN++] = pass[j];
+            if (visited.insert(pass[j]).second) fresh.push_back(pass[j]);
+        }
+        if (size_EN == B) break;
+    }
+    if (rows_read) *rows_read = rows;
+    return size_EN;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Squared L2 distance in fp32, fixed order.  The d floats are cut into 4-float groups; group g
 // goes to partial sum g mod 8; each partial sum takes its groups in increasing g, elements in
 // increasing index, acc = fma(x - q, x - q, acc); then the 8 partial sums are combined by a
@@ -241,6 +281,7 @@ struct Params {
     int warp;        // chunk width of Alg. 4 (32; any value gives the same EN list)
     int no_hotspot;  // ablation: scan all H layers
     int exact_below; // ranges of at most this many objects are answered by the exact scan too (0: off)
+    int eager_hash;  // ablation: visited test inside the predicate of Alg. 4 instead of after it
 };
 
 // status bits
@@ -290,6 +331,7 @@ void search_one(const Index& ix, const float* v_q, int32_t lo, int32_t hi, int k
         if ((int)pool.size() > ef_s) pool.resize(ef_s);
         std::vector<uint32_t> EN(P.B > 0 ? P.B : 1);
         std::vector<Cand> fresh;
+        std::vector<uint32_t> fresh_ids;
         for (;;) {                                                            // line 7
             // line 17 (and line 6): first pool position whose flag is 0
             int i = 0;
@@ -299,8 +341,11 @@ void search_one(const Index& ix, const float* v_q, int32_t lo, int32_t hi, int k
             uint32_t u = pool[i].id;                                          // line 8
             pool[i].flag = 1;                                                 // line 9
             int rows = 0;
-            int cnt = en_identification(ix.enc + (int64_t)u * ix.H * ix.m, ix.m, l_q, r_q,
-                                        L_start, L_end, P.B, P.warp, EN.data(), &rows);   // line 10
+            int cnt = P.eager_hash
+                ? en_identification_eager(ix.enc + (int64_t)u * ix.H * ix.m, ix.m, l_q, r_q, L_start, L_end,
+                                          P.B, P.warp, visited, EN.data(), fresh_ids, &rows)
+                : en_identification(ix.enc + (int64_t)u * ix.H * ix.m, ix.m, l_q, r_q,
+                                    L_start, L_end, P.B, P.warp, EN.data(), &rows);       // line 10
             ++n_exp; n_rows += rows; n_en += cnt;
             if (trace && trace_ok && (int64_t)trace->size() + 66 > trace_cap - 1) trace_ok = false;   // 66 = header + 64 entries
             if (trace && trace_ok) {
@@ -309,9 +354,9 @@ void search_one(const Index& ix, const float* v_q, int32_t lo, int32_t hi, int k
                 for (int j = 0; j < cnt; ++j) trace->push_back(EN[j]);
             }
             fresh.clear();                                                    // line 11
-            for (int j = 0; j < cnt; ++j) {                                   // line 12
-                uint32_t v = EN[j];
-                if (visited.insert(v).second) {                               // line 13
+            for (int j = 0; j < (P.eager_hash ? (int)fresh_ids.size() : cnt); ++j) {   // line 12
+                uint32_t v = P.eager_hash ? fresh_ids[j] : EN[j];
+                if (P.eager_hash || visited.insert(v).second) {               // line 13
                     fresh.push_back(Cand{dist2_canonical(v_q, ix.vectors + (int64_t)v * ix.d_pad, ix.d_pad), v, 0});
                     ++n_dist;                                                 // line 14
                 }
@@ -368,11 +413,11 @@ int frog_oracle_search(const int32_t* sorted_attr, const int32_t* rank2id, const
                        const uint32_t* enc, int64_t n, int d_pad, int H, int m,
                        const float* queries, const int32_t* lo, const int32_t* hi, int64_t nq,
                        int k, int ef_s, int epn, int B, int max_iters, uint64_t seed, int warp,
-                       int no_hotspot, int exact_below,
+                       int no_hotspot, int exact_below, int eager_hash,
                        int32_t* out_ids, float* out_dists, uint32_t* status, uint32_t* stats,
                        uint32_t* trace_out, int64_t trace_cap, int threads) {
     Index ix{sorted_attr, rank2id, vectors, enc, n, d_pad, H, m};
-    Params P{epn, B, max_iters, seed, warp, no_hotspot, exact_below};
+    Params P{epn, B, max_iters, seed, warp, no_hotspot, exact_below, eager_hash};
     int used = 1;
 #ifdef _OPENMP
     omp_set_num_threads(threads > 0 ? threads : omp_get_num_procs());   // <= 0: all cores

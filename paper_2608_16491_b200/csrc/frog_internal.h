@@ -35,6 +35,7 @@ struct FrogSearchArgs {
     const int32_t* lo;
     const int32_t* hi;
     int nq, k, ef_s, epn, B, max_iters, no_hotspot, hash_bits;
+    int exact_w;               // ranges of at most this many objects are scanned exactly (>= ef_s)
     unsigned long long seed;
     int32_t* out_ids;
     float* out_dists;

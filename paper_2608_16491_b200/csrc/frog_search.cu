@@ -248,8 +248,8 @@ frog_search_kernel(const FrogSearchArgs A) {
 
         if (w <= 0) {
             st |= FROG_ST_EMPTY;
-        } else if (w <= A.ef_s) {
-            // every valid object enters the pool: exact answer
+        } else if (w <= A.exact_w) {
+            // every valid object is evaluated, the pool keeps the ef_s nearest: exact answer
             st |= FROG_ST_EXACT;
             for (int b0 = 0; b0 < w; b0 += 32) {
                 const int cnt = min(32, w - b0);
@@ -567,6 +567,7 @@ int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in
     if (P.visited != FROG_VISITED_AUTO && P.visited != FROG_VISITED_BITMAP && P.visited != FROG_VISITED_HASH)
         return FROG_ERR_INVALID_ARG;
     if (P.storage != FROG_STORAGE_F32 && P.storage != FROG_STORAGE_F16) return FROG_ERR_INVALID_ARG;
+    if (P.exact_below < 0 || P.reserved != 0) return FROG_ERR_INVALID_ARG;
     if (P.storage == FROG_STORAGE_F16 && !ix->d_vectors_h) return FROG_ERR_INVALID_ARG;   // not enabled on this index
     (void)ix;
     *out = P;
@@ -678,6 +679,7 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     A.B = P.budget;
     A.max_iters = P.max_iters;
     A.no_hotspot = P.no_hotspot;
+    A.exact_w = P.exact_below > beam_width ? P.exact_below : beam_width;
     A.hash_bits = P.hash_bits;
     A.seed = P.seed;
     A.out_ids = out_ids;
@@ -804,6 +806,7 @@ extern "C" int frog_search_static(const frog_index_t* index, const float* querie
     A.B = P.budget;
     A.max_iters = P.max_iters;
     A.no_hotspot = P.no_hotspot;
+    A.exact_w = P.exact_below > beam_width ? P.exact_below : beam_width;
     A.hash_bits = P.hash_bits;
     A.seed = P.seed;
     A.out_ids = out_ids;

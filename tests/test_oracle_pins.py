@@ -385,6 +385,46 @@ def test_search_counters_and_trace_are_consistent(tiny_runs):
         assert n_rows <= n_exp * ix.H and n_dist <= 16 + n_en
 
 
+def test_eager_hash_check_ablation(tiny_runs):
+    """Eager form of the hash check (visited test inside the predicate of Alg. 4).  (a) When the
+    budget never binds (B >= H*m) it evaluates the same vertices as the lazy form, so ids,
+    distances, expansions and distance counts coincide with the pinned lazy search.  (b) With
+    the default budget, replaying the trace: no EN entry was evaluated before its expansion,
+    repeats occur only inside one EN list, and the distance count is the number of distinct ids."""
+    wl, ix, _, _, runs = tiny_runs
+    big = ix.H * ix.m
+    lazy = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 64, B=big)
+    eager = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 64, B=big, eager_hash=True)
+    assert np.array_equal(lazy.ids, eager.ids) and np.array_equal(lazy.dists, eager.dists)
+    assert np.array_equal(lazy.stats[:, [0, 3]], eager.stats[:, [0, 3]])
+    assert eager.stats[:, 2].sum() < lazy.stats[:, 2].sum()          # fewer admitted slots
+
+    res = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 64, eager_hash=True, trace_cap=8192)
+    searched = 0
+    for q in range(wl.nq):
+        if res.status[q] & (oracle.ST_EXACT | oracle.ST_EMPTY):
+            continue
+        searched += 1
+        l, r = oracle.rank_interval(ix.sorted_attr, int(wl.lo[q]), int(wl.hi[q]))
+        seen = {oracle.entry_point(0, l, r, j) for j in range(16)}
+        tr = res.trace[q]
+        pos, ln, n_en = 1, int(tr[0]), 0
+        while pos < 1 + ln:
+            cnt = int(tr[pos + 1])
+            en = [int(x) for x in tr[pos + 2: pos + 2 + cnt]]
+            assert cnt <= 16 and not (set(en) & seen)
+            seen |= set(en)
+            n_en += cnt
+            pos += 2 + cnt
+        assert n_en == int(res.stats[q, 2]) and len(seen) == int(res.stats[q, 3])
+    assert searched > 50
+    # the eager form spends its budget on unevaluated vertices only: at least as many distances
+    # per expansion as the lazy form
+    base = runs[64]
+    m = (base.stats[:, 0] > 0)
+    assert (res.stats[m, 3] / res.stats[m, 0]).mean() >= (base.stats[m, 3] / base.stats[m, 0]).mean()
+
+
 def test_recall_improves_with_beam_and_is_high(tiny_runs):
     wl, ix, gt_ids, _, runs = tiny_runs
     rec = {ef: oracle.recall(res.ids, gt_ids) for ef, res in runs.items()}
