@@ -75,7 +75,9 @@ typedef struct {
                            scanning their contiguous rank slab (exact, status FROG_ST_EXACT) instead of
                            the graph search; 0 = default: only ranges that fit the pool.  Not in the
                            paper, whose smallest ranges hold thousands of objects (Sec. 8.1.2) */
-    int32_t reserved;   /* must be 0 */
+    int32_t eager_hash; /* nonzero: ablation of the lazy hash check (Sec. 6.2): the visited test moves into
+                           the predicate of Alg. 4, so evaluated ids neither take a slot nor consume
+                           budget.  Bitmap visited form, fp32 storage and no trace only */
 } frog_params_t;
 
 /* Vector storage read by the search.  F32 (default): the index's fp32 rows.  F16: an fp16 copy made

@@ -46,7 +46,7 @@ class Params(C.Structure):
     _fields_ = [("epn", C.c_int32), ("budget", C.c_int32), ("max_iters", C.c_int32),
                 ("no_hotspot", C.c_int32), ("seed", C.c_uint64), ("hash_bits", C.c_int32),
                 ("visited", C.c_int32), ("storage", C.c_int32), ("debug_flags", C.c_int32),
-                ("exact_below", C.c_int32), ("reserved", C.c_int32)]
+                ("exact_below", C.c_int32), ("eager_hash", C.c_int32)]
 
 
 class BuildParams(C.Structure):

@@ -41,7 +41,7 @@ constexpr int WARPS_PER_CTA = FROG_WARPS_PER_CTA;
 #ifndef FROG_EVAL_INLINE
 #define FROG_EVAL_INLINE __noinline__
 #endif
-constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2;
+constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2, MODE_EAGER = 3;   // EAGER: FAST with the eager hash check
 
 #ifndef FROG_ENC_PREFETCH
 #define FROG_ENC_PREFETCH 1   // 0: off, 1: prefetch the predicted vertex's ENC lines
@@ -158,7 +158,8 @@ __device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows
 }
 
 template <int EPL, int MODE, bool BITMAP, bool F16, int ROWB = 0>
-__global__ void __launch_bounds__(WARPS_PER_CTA * 32, MODE == MODE_FAST ? (EPL <= 4 ? FROG_MINB : FROG_MINB_BIG) : 1)
+__global__ void __launch_bounds__(WARPS_PER_CTA * 32,
+                                  (MODE == MODE_FAST || MODE == MODE_EAGER) ? (EPL <= 4 ? FROG_MINB : FROG_MINB_BIG) : 1)
 frog_search_kernel(const FrogSearchArgs A) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int lane = lane_id();
@@ -243,7 +244,7 @@ frog_search_kernel(const FrogSearchArgs A) {
         uint32_t st = 0, n_exp = 0, n_rows = 0, n_en = 0, n_dist = 0, forgets = 0;
         uint32_t trace_len = 0;
         bool trace_ok = true;
-        uint32_t* trace_row = (MODE != MODE_FAST) ? A.trace + (size_t)q * A.trace_cap : nullptr;
+        uint32_t* trace_row = (MODE == MODE_TRACE || MODE == MODE_PROFILE) ? A.trace + (size_t)q * A.trace_cap : nullptr;
         __syncwarp();
 
         if (w <= 0) {
@@ -310,6 +311,32 @@ frog_search_kernel(const FrogSearchArgs A) {
                 const bool rec_ok = (MODE == MODE_TRACE) && trace_ok && (trace_len + 66 <= (uint32_t)A.trace_cap - 1);
                 int cnt = 0, scanned = 0;
                 ns = 0;
+                if (MODE == MODE_EAGER) {
+                    // Ablation: the visited test is part of the predicate.  One 32-entry chunk at a
+                    // time: every lane tests against the bitmap as the previous chunk left it, the
+                    // admitted prefix sets its bits (a second copy of an id inside the chunk is
+                    // admitted, finds the bit set and is dropped).
+                    for (int c0 = 0; c0 < total && cnt < A.B; c0 += 32) {
+                        uint32_t v = BOT;
+                        if (c0 + lane < total) v = FROG_ENC_LD(hot + c0 + lane);
+                        const bool in_range = (v - (uint32_t)l_q) <= span;
+                        const uint32_t bit = 1u << (v & 31);
+                        uint32_t word = 0xFFFFFFFFu;
+                        if (in_range) word = __ldcg(bitmap + (v >> 5));
+                        const bool pred = (word & bit) == 0;
+                        const uint32_t M = __ballot_sync(FULL, pred);
+                        const int a = min(__popc(M), A.B - cnt);
+                        const bool adm = pred && __popc(M & lt_mask) < a;
+                        uint32_t old = 0xFFFFFFFFu;
+                        if (adm) old = atomicOr(bitmap + (v >> 5), bit);
+                        const bool keep = (old & bit) == 0;
+                        const uint32_t K = __ballot_sync(FULL, keep);
+                        if (keep) S.cand[ns + __popc(K & lt_mask)] = v;
+                        ns += __popc(K);
+                        cnt += a;
+                        scanned = min(total, c0 + 32);
+                    }
+                } else
                 for (int c0 = 0; c0 < total && cnt < A.B; c0 += 64) {
                     uint32_t v0 = BOT, v1 = BOT;
                     if (c0 + lane < total) v0 = FROG_ENC_LD(hot + c0 + lane);
@@ -492,8 +519,12 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
         fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, false, false>(beam_width, &pool_slots)
            : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, false, false>(beam_width, &pool_slots)
                                   : pick_kernel<MODE_FAST, false, false>(beam_width, &pool_slots);
+    if (P.eager_hash) {
+        if (!bitmap || f16 || mode != MODE_FAST) return FROG_ERR_UNSUPPORTED;
+        fn = pick_kernel<MODE_EAGER, true, false>(beam_width, &pool_slots);
+    }
     // common shape with the geometry fixed at compile time: fp32 rows of 512 bytes (d = 125..128)
-    if (mode == MODE_FAST && bitmap && !f16 && ix->info.d_pad == 128) {
+    if (mode == MODE_FAST && bitmap && !f16 && !P.eager_hash && ix->info.d_pad == 128) {
         if (beam_width <= 32) fn = frog_search_kernel<1, MODE_FAST, true, false, 512>;
         else if (beam_width <= 64) fn = frog_search_kernel<2, MODE_FAST, true, false, 512>;
         else if (beam_width <= 128) fn = frog_search_kernel<4, MODE_FAST, true, false, 512>;
@@ -567,7 +598,7 @@ int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in
     if (P.visited != FROG_VISITED_AUTO && P.visited != FROG_VISITED_BITMAP && P.visited != FROG_VISITED_HASH)
         return FROG_ERR_INVALID_ARG;
     if (P.storage != FROG_STORAGE_F32 && P.storage != FROG_STORAGE_F16) return FROG_ERR_INVALID_ARG;
-    if (P.exact_below < 0 || P.reserved != 0) return FROG_ERR_INVALID_ARG;
+    if (P.exact_below < 0) return FROG_ERR_INVALID_ARG;
     if (P.storage == FROG_STORAGE_F16 && !ix->d_vectors_h) return FROG_ERR_INVALID_ARG;   // not enabled on this index
     (void)ix;
     *out = P;

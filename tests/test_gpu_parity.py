@@ -98,15 +98,18 @@ def test_tiny_plain_call_equals_ex_call(libs, tiny_gpu):
                                     dict(budget=64), dict(budget=64, visited=2), dict(budget=40, no_hotspot=1),
                                     dict(no_hotspot=1), dict(seed=12345), dict(max_iters=7),
                                     dict(epn=7, budget=9, seed=3), dict(exact_below=700),
-                                    dict(exact_below=3000, visited=2, budget=32)])
+                                    dict(exact_below=3000, visited=2, budget=32), dict(eager_hash=1),
+                                    dict(eager_hash=1, budget=64), dict(eager_hash=1, budget=5, epn=3),
+                                    dict(eager_hash=1, no_hotspot=1, budget=33)])
 def test_tiny_parameter_variants(libs, tiny_gpu, params):
     wl, ix, gix = tiny_gpu
     params = dict(params)
     okw = dict(epn=params.get("epn", 16), B=params.get("budget", 16), seed=params.get("seed", 0),
                no_hotspot=bool(params.get("no_hotspot", 0)), max_iters=params.get("max_iters", 0),
-               exact_below=params.get("exact_below", 0))
-    ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 48, trace_cap=20000, **okw)
-    got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, wl.k, 48, trace_cap=20000, **params)
+               exact_below=params.get("exact_below", 0), eager_hash=bool(params.get("eager_hash", 0)))
+    cap = 0 if params.get("eager_hash") else 20000      # the eager ablation has no trace kernel
+    ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 48, trace_cap=cap, **okw)
+    got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, wl.k, 48, trace_cap=cap, **params)
     _assert_parity(got, ref, slots=_default_slots(48))
 
 
@@ -158,6 +161,8 @@ def test_empty_batch_and_argument_errors(libs, tiny_gpu):
         gix.search(q, lo, hi, 10, 32, params=libs.Params(budget=65))
     with pytest.raises(libs.FrogError):
         gix.search(q, lo, hi, 10, 32, params=libs.Params(exact_below=-1))
+    with pytest.raises(libs.FrogError):                  # the ablation exists for the bitmap form only
+        gix.search(q, lo, hi, 10, 32, params=libs.Params(eager_hash=1, visited=libs.VISITED_HASH))
     # a failed call leaves the index usable
     ids, _ = gix.search(q, lo, hi, 10, 32)
     torch.cuda.synchronize()
