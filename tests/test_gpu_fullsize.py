@@ -13,11 +13,12 @@ pytestmark = pytest.mark.gpu
 
 torch = pytest.importorskip("torch")
 
-BEAM, BUDGET = 112, 32
+POINTS = [(44, 64), (112, 32)]     # (beam_width, budget): the bench point and the best B = 32 point
 
 
-@pytest.fixture(scope="module")
-def full(libs):
+@pytest.fixture(scope="module", params=POINTS, ids=lambda p: f"ef{p[0]}_B{p[1]}")
+def full(libs, request):
+    BEAM, BUDGET = request.param
     if os.environ.get("FROG_SKIP_FULLSIZE") == "1":
         pytest.skip("FROG_SKIP_FULLSIZE=1")
     import bench
@@ -32,7 +33,7 @@ def full(libs):
     stats = torch.zeros((wl.nq, 4), dtype=torch.int32, device="cuda")
     ids, dists = gix.search(q, lo, hi, wl.k, BEAM, params=libs.Params(budget=BUDGET), status=status, stats=stats)
     torch.cuda.synchronize()
-    out = dict(wl=wl, path=path, gix=gix, q=q, lo=lo, hi=hi, ids=ids.cpu().numpy(), dists=dists.cpu().numpy(),
+    out = dict(beam=BEAM, budget=BUDGET, wl=wl, path=path, gix=gix, q=q, lo=lo, hi=hi, ids=ids.cpu().numpy(), dists=dists.cpu().numpy(),
                status=status.cpu().numpy().view(np.uint32), stats=stats.cpu().numpy().view(np.uint32))
     yield out
     gix.close()
@@ -43,7 +44,7 @@ def test_sampled_queries_equal_the_oracle(full):
     ix = oracle.load_index(full["path"])
     rng = np.random.default_rng(7)
     sample = np.sort(rng.choice(wl.nq, size=400, replace=False))
-    ref = oracle.search(ix, wl.queries[sample], wl.lo[sample], wl.hi[sample], wl.k, BEAM, B=BUDGET)
+    ref = oracle.search(ix, wl.queries[sample], wl.lo[sample], wl.hi[sample], wl.k, full["beam"], B=full["budget"])
     assert np.array_equal(full["ids"][sample], ref.ids)                    # bit-exact ids
     fin = np.isfinite(ref.dists)
     assert np.allclose(full["dists"][sample][fin], ref.dists[fin], rtol=1e-4, atol=0)
@@ -97,8 +98,8 @@ def test_static_entry_point_at_full_size(full, libs):
     wl = full["wl"]
     out_ids = torch.empty((wl.nq, wl.k), dtype=torch.int32, device="cuda")
     out_d = torch.empty((wl.nq, wl.k), dtype=torch.float32, device="cuda")
-    full["gix"].search_static(full["q"], full["lo"], full["hi"], wl.k, BEAM, out_ids=out_ids, out_dists=out_d,
-                              params=libs.Params(budget=BUDGET))
+    full["gix"].search_static(full["q"], full["lo"], full["hi"], wl.k, full["beam"], out_ids=out_ids, out_dists=out_d,
+                              params=libs.Params(budget=full["budget"]))
     torch.cuda.synchronize()
     assert np.array_equal(out_ids.cpu().numpy(), full["ids"])
 
@@ -108,9 +109,9 @@ ALL = os.environ.get("FROG_FULLSIZE_ALL") == "1"
 
 
 @pytest.mark.skipif(not ALL, reason="set FROG_FULLSIZE_ALL=1 to run the 1M x 96, 10M x 96 and 1M x 768 workloads")
-@pytest.mark.parametrize("name,k,beam", [("deep1m", 10, 128), ("text", 10, 128), ("deep10m", 10, 128),
-                                         ("deep10m", 100, 128)])
-def test_other_workloads_at_full_size(libs, name, k, beam):
+@pytest.mark.parametrize("name,k,beam,BUDGET", [("deep1m", 10, 128, 32), ("deep1m", 10, 64, 64), ("text", 10, 128, 32),
+                                                ("text", 10, 64, 64), ("deep10m", 10, 64, 64), ("deep10m", 100, 128, 32)])
+def test_other_workloads_at_full_size(libs, name, k, beam, BUDGET):
     import bench
     import datagen
     wl = datagen.make_workload(name, k=k)
@@ -140,7 +141,7 @@ def test_other_workloads_at_full_size(libs, name, k, beam):
         gt, _, _ = oracle.exact_slab(ix, wl.queries[sample], wl.lo[sample], wl.hi[sample], k, mode=0)
         rec_gpu, rec_ref = oracle.recall(ids[sample], gt), oracle.recall(ref.ids, gt)
         assert abs(rec_gpu - rec_ref) <= 0.005
-        print(f"[fullsize] {name} k={k} beam={beam}: build {secs:.1f}s recall@{k} {rec_gpu:.4f} (sample of 200)")
+        print(f"[fullsize] {name} k={k} beam={beam} B={BUDGET}: build {secs:.1f}s recall@{k} {rec_gpu:.4f} (sample of 200)")
         # whole batch: range, order, padding
         valid = ids >= 0
         a = wl.attrs[np.where(valid, ids, 0)]
@@ -155,7 +156,7 @@ def test_other_workloads_at_full_size(libs, name, k, beam):
         assert np.array_equal(e_ids.cpu().numpy(), r_ids) and np.array_equal(e_d.cpu().numpy(), r_d)
     finally:
         gix.close()
-        # do not leave multi-gigabyte files behind on a shared machine (the 10M index is reused by the
-        # k = 100 case that follows it in the parameter list)
-        if os.path.getsize(path) > (4 << 30) and not (name == "deep10m" and k == 10):
+        # do not leave multi-gigabyte files behind on a shared machine (an index is reused by the case
+        # of the same workload that follows it in the parameter list)
+        if os.path.getsize(path) > (4 << 30) and (name, beam, BUDGET) in (("text", 64, 64), ("deep10m", 128, 32)):
             os.remove(path)
