@@ -115,7 +115,7 @@ def test_tiny_parameter_variants(libs, tiny_gpu, params):
 
 def test_k_equals_beam_and_k_one(libs, tiny_gpu):
     wl, ix, gix = tiny_gpu
-    for k, ef in ((32, 32), (1, 16), (100, 128), (64, 64)):
+    for k, ef in ((32, 32), (1, 16), (100, 128), (64, 64), (256, 512), (512, 512)):
         ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef)
         got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, k, ef)
         _assert_parity(got, ref, slots=_default_slots(ef))
@@ -133,6 +133,41 @@ def test_edge_ranges(libs, tiny_gpu):
     _assert_parity(got, ref, check_dist_count=False)
     assert ref.status[0] & oracle.ST_EMPTY and ref.status[1] & oracle.ST_EMPTY
     assert ref.status[4] & oracle.ST_EXACT and not (ref.status[5] & oracle.ST_EXACT)
+
+
+def test_side_stream_and_back_to_back_calls(libs, tiny_gpu):
+    """The call is asynchronous on the caller's stream: two searches queued back to back on a side
+    stream (the second overwrites the scratch of the first) give the answers of separate calls."""
+    wl, ix, gix = tiny_gpu
+    q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        a_ids, a_d = gix.search(q, lo, hi, wl.k, 32, stream=side, params=libs.Params(budget=64))
+        b_ids, b_d = gix.search(q, lo, hi, wl.k, 96, stream=side)
+    side.synchronize()
+    ref_a = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 32, B=64)
+    ref_b = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 96)
+    assert np.array_equal(a_ids.cpu().numpy(), ref_a.ids) and np.array_equal(a_d.cpu().numpy(), ref_a.dists)
+    assert np.array_equal(b_ids.cpu().numpy(), ref_b.ids) and np.array_equal(b_d.cpu().numpy(), ref_b.dists)
+
+
+def test_non_finite_queries_terminate(libs, tiny_gpu):
+    """Non-finite query components: the results are unspecified, but the call returns, every
+    reported id lies in the query's range and no wait ran into its limit."""
+    wl, ix, gix = tiny_gpu
+    Q = wl.queries[:64].copy()
+    Q[0::4, 3] = np.nan
+    Q[1::4, :] = np.inf
+    Q[2::4, 5] = -np.inf
+    Q[3::4, :] = 3.0e38
+    got = _gpu_search(libs, gix, Q, wl.lo[:64], wl.hi[:64], wl.k, 48, budget=64)
+    ids, dists, status, stats, _ = got
+    assert not (status & 32).any()
+    assert np.all(stats[:, 0] <= 16 * 48)                                  # the expansion cap held
+    valid = ids >= 0
+    a = wl.attrs[np.where(valid, ids, 0)]
+    assert np.all(~valid | ((a >= wl.lo[:64, None]) & (a <= wl.hi[:64, None])))
 
 
 def test_small_visited_table_changes_work_not_results(libs, tiny_gpu):
