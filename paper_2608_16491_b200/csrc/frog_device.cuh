@@ -391,6 +391,105 @@ __device__ __forceinline__ float staged_dist2_flex(const void* __restrict__ rows
     return out;
 }
 
+// The same computation as staged_dist2_flex with the stage buffer split into two halves, each with
+// its own mbarrier: while the teams reduce the rows of one half, the copies of the next group of
+// rows are already landing in the other, so the arithmetic hides behind the copy latency.  A
+// group is up to 8 rows (4 for 512-byte slots: one row per team); a row longer than STAGE_CHUNK is
+// taken in column chunks, one chunk of every row of the group per step.  bar[0], bar[1] are the
+// two mbarriers; `phases` holds their parities in bits 0 and 1.
+template <bool F16, int ROWB = 0>
+__device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows, int row_bytes, int slot_bytes,
+                                                   const float4* qs, float4* stage, uint64_t* bar,
+                                                   uint32_t& phases, bool& ok, uint32_t my_rank, int ns, int lane) {
+    if (ROWB > 0) {
+        row_bytes = ROWB;
+        slot_bytes = ROWB >= STAGE_CHUNK ? STAGE_CHUNK : ROWB;     // ROWB is a power of two when below 512
+    }
+    constexpr int HALF = FROG_STAGE_ROWS * STAGE_CHUNK / 2;
+    constexpr int GROUP_BYTES = F16 ? 8 : 16;             // 4 elements
+    const int rph = (HALF / slot_bytes) > 8 ? 8 : (HALF / slot_bytes);     // rows per half
+    const int chunks = (row_bytes + STAGE_CHUNK - 1) / STAGE_CHUNK;
+    const int steps = ((ns + rph - 1) / rph) * chunks;
+    const int team = lane >> 3, sub = lane & 7;
+    int ig = 0, ic = 0;                                   // group and chunk of the next step to issue
+    auto issue = [&](int s) {
+        const int r0 = ig * rph, nrows = min(rph, ns - r0);
+        const int c0 = ic * STAGE_CHUNK, cbytes = min(STAGE_CHUNK, row_bytes - c0);
+        uint64_t* b = bar + (s & 1);
+        if (lane == 0) mbar_expect_tx(b, (uint32_t)(nrows * cbytes));
+        __syncwarp();
+        const uint32_t copy_rank = __shfl_sync(FULL, my_rank, (r0 + lane) & 31);
+        if (lane < nrows)
+            tma_load_1d(reinterpret_cast<char*>(stage) + (s & 1) * HALF + lane * slot_bytes,
+                        reinterpret_cast<const char*>(rows) + (size_t)copy_rank * (size_t)row_bytes + c0,
+                        (uint32_t)cbytes, b);
+        if (++ic == chunks) { ic = 0; ++ig; }
+    };
+    issue(0);
+    if (steps > 1) issue(1);
+    float out = 0.f, acc0 = 0.f, acc1 = 0.f;
+    int g = 0, c = 0;
+#pragma unroll 1
+    for (int s = 0; s < steps; ++s) {
+        const int h = s & 1;
+        ok = mbar_wait(bar + h, (phases >> h) & 1u) && ok;
+        phases ^= 1u << h;
+        const int r0 = g * rph, nrows = min(rph, ns - r0);
+        const int c0 = c * STAGE_CHUNK, cbytes = min(STAGE_CHUNK, row_bytes - c0);
+        const int g_lo = c0 / GROUP_BYTES, g_n = cbytes / GROUP_BYTES;
+        const char* half = reinterpret_cast<const char*>(stage) + h * HALF;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int r = i * 4 + team;
+            if ((i == 0 || rph > 4) && r < nrows) {
+                const char* xrow = half + r * slot_bytes;
+                float a = i == 0 ? acc0 : acc1;
+#pragma unroll 4
+                for (int gg = sub; gg < g_n; gg += 8) {
+                    float4 x;
+                    if (F16) {
+                        const uint2 raw = *reinterpret_cast<const uint2*>(xrow + gg * 8);
+                        const float2 lo2 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+                        const float2 hi2 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+                        x = make_float4(lo2.x, lo2.y, hi2.x, hi2.y);
+                    } else {
+                        x = *reinterpret_cast<const float4*>(xrow + gg * 16);
+                    }
+                    const float4 q = qs[g_lo + gg];
+                    float t;
+                    t = x.x - q.x; a = fmaf(t, t, a);
+                    t = x.y - q.y; a = fmaf(t, t, a);
+                    t = x.z - q.z; a = fmaf(t, t, a);
+                    t = x.w - q.w; a = fmaf(t, t, a);
+                }
+                if (i == 0) acc0 = a; else acc1 = a;
+            }
+        }
+        if (c == chunks - 1) {
+            const int src = ((lane - r0) & 3) << 3;         // team that summed this lane's row
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                if ((i == 0 || rph > 4) && i * 4 < nrows) {
+                    float a = i == 0 ? acc0 : acc1;
+                    a = a + __shfl_xor_sync(FULL, a, 4);
+                    a = a + __shfl_xor_sync(FULL, a, 2);
+                    a = a + __shfl_xor_sync(FULL, a, 1);
+                    const float v = __shfl_sync(FULL, a, src);
+                    if (lane >= r0 && ((lane - r0) >> 2) == i && lane - r0 < nrows) out = v;
+                }
+            }
+            acc0 = acc1 = 0.f;
+            c = 0;
+            ++g;
+        } else {
+            ++c;
+        }
+        __syncwarp();                                       // every lane is done reading this half
+        if (s + 2 < steps) issue(s + 2);
+    }
+    return out;
+}
+
 // two smallest values seen by a lane
 __device__ __forceinline__ void track2(int& m1, int& m2, int p) {
     if (p < m1) { m2 = m1; m1 = p; }
@@ -413,7 +512,7 @@ __device__ __forceinline__ uint32_t first_two(int m1, int m2) {
 // hold the pool keys (lane l owns positions l, l+32, ...).  A new key equal to a pool key (a vertex
 // the visited table forgot) or to an earlier new key is discarded.  Returns the positions of the
 // first and of the second entry whose flag is 0, packed as first | second << 16 (0xFFFF = none).
-template <int EPL>
+template <int EPL, bool UNIQUE = false>
 __device__ __forceinline__ uint32_t merge_batch(uint64_t* pool, uint64_t my_key, int ef_s, int lane) {
     uint64_t pk[EPL];
 #pragma unroll
@@ -440,18 +539,19 @@ __device__ __forceinline__ uint32_t merge_batch(uint64_t* pool, uint64_t my_key,
     for (uint32_t msk = have; msk; msk &= msk - 1) {
         const int j = __ffs(msk) - 1;
         const uint64_t x = ((uint64_t)__shfl_sync(FULL, my_hi, j) << 32) | __shfl_sync(FULL, my_lo, j);
-        // copies: of a pool key, or of a new key held by a lower lane
-        bool eq = (x == mk) && (lane < j);
+        // copies: of a pool key, or of a new key held by a lower lane (UNIQUE: the caller
+        // guarantees there are none, e.g. an exact visited set)
+        bool eq = !UNIQUE && (x == mk) && (lane < j);
         bool lt[EPL];
         int cnt_above = 0;
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const uint64_t p = pk[e] | 1ull;
             lt[e] = x < p;
-            eq = eq || (x == p);
+            if (!UNIQUE) eq = eq || (x == p);
             cnt_above += __popc(__ballot_sync(FULL, lt[e]));
         }
-        if (__any_sync(FULL, eq)) {
+        if (!UNIQUE && __any_sync(FULL, eq)) {
             if (lane == j) dropped = true;
             continue;
         }

@@ -38,6 +38,9 @@ constexpr int WARPS_PER_CTA = FROG_WARPS_PER_CTA;
 #ifndef FROG_MINB_BIG
 #define FROG_MINB_BIG 4       // the same for pools above 128 entries
 #endif
+#ifndef FROG_UNIQUE_MERGE
+#define FROG_UNIQUE_MERGE 1   // bitmap visited set: keys reaching the merge are distinct, skip the copy test
+#endif
 #ifndef FROG_EVAL_INLINE
 #define FROG_EVAL_INLINE __noinline__
 #endif
@@ -54,18 +57,19 @@ constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2, MODE_EAGER = 3;  
 #endif
 constexpr int STAGE_BYTES = FROG_STAGE_ROWS * STAGE_CHUNK;
 
-// per-warp shared memory: pool | candidate list | mbarrier, its phase, a failure flag | query | stage | hash
+// per-warp shared memory: pool | candidate list | two mbarriers, their parities, a failure flag | query | stage | hash
 struct WarpSmem {
     uint64_t* pool;
     uint32_t* cand;
-    uint64_t* bar;       // bar[0] = mbarrier; the two words after it: phase parity, copy-timeout flag
+    uint64_t* bar;       // bar[0], bar[1] = mbarriers of the two stage halves; the two words after them:
+                         // their phase parities (bits 0, 1) and the copy-timeout flag; 32 bytes in all
     float4* q;
     float4* stage;
     uint32_t* hash;
 };
 
 inline size_t warp_smem_bytes(int pool_slots, int q_len, int hash_bits, bool bitmap) {
-    return (size_t)pool_slots * 8 + 64 * 4 + 16 + (size_t)q_len * 4 + STAGE_BYTES +
+    return (size_t)pool_slots * 8 + 64 * 4 + 32 + (size_t)q_len * 4 + STAGE_BYTES +
            (bitmap ? 0 : ((size_t)4 << hash_bits));
 }
 inline int query_len(int d) { return (d + 7) / 8 * 8; }
@@ -98,7 +102,7 @@ __device__ __forceinline__ bool visited_test_and_set(const WarpSmem& S, uint32_t
 // Distances of the ns <= 32 ranks listed in cand[0..ns) and their merge into the pool (Alg. 2
 // lines 14-17).  Returns the first unexpanded pool position.  Kept out of line: it is called from
 // three places of the kernel and inlining every copy costs registers and instruction cache.
-template <int EPL, bool F16, int ROWB>
+template <int EPL, bool F16, int ROWB, bool UNIQUE>
 __device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows, int row_bytes, int slot_bytes,
                                                    int rows_per_pass, int ef_s,
                                                    uint64_t* pool, const uint32_t* cand, uint64_t* bar,
@@ -124,11 +128,11 @@ __device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows
     }
     float d2 = 0.f;
     if (ns > 0) {
-        uint32_t* bar_words = reinterpret_cast<uint32_t*>(bar + 1);
+        uint32_t* bar_words = reinterpret_cast<uint32_t*>(bar + 2);
         __syncwarp();                       // lane 0's update of the parity in the previous call
         uint32_t phase = bar_words[0];
         bool ok = true;
-        d2 = staged_dist2_flex<F16, ROWB>(rows, row_bytes, slot_bytes, rows_per_pass, qs, stage, bar, phase, ok, id, ns, lane);
+        d2 = staged_dist2_pipe<F16, ROWB>(rows, row_bytes, slot_bytes, qs, stage, bar, phase, ok, id, ns, lane);
         __syncwarp();                       // every lane has read the old parity
         if (lane == 0) {
             bar_words[0] = phase;
@@ -154,7 +158,7 @@ __device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows
         }
     }
 #endif
-    return (int)merge_batch<EPL>(pool, key, ef_s, lane);
+    return (int)merge_batch<EPL, UNIQUE>(pool, key, ef_s, lane);
 }
 
 template <int EPL, int MODE, bool BITMAP, bool F16, int ROWB = 0>
@@ -166,19 +170,20 @@ frog_search_kernel(const FrogSearchArgs A) {
     const int warp = threadIdx.x >> 5;
     constexpr int POOL = 32 * EPL;
     const int hash_slots = BITMAP ? 0 : (1 << A.hash_bits);
-    const size_t per_warp = (size_t)POOL * 8 + 64 * 4 + 16 + (size_t)A.q_len * 4 + STAGE_BYTES + (size_t)hash_slots * 4;
+    const size_t per_warp = (size_t)POOL * 8 + 64 * 4 + 32 + (size_t)A.q_len * 4 + STAGE_BYTES + (size_t)hash_slots * 4;
     unsigned char* base = smem_raw + per_warp * warp;
     WarpSmem S;
     S.pool = reinterpret_cast<uint64_t*>(base);
     S.cand = reinterpret_cast<uint32_t*>(S.pool + POOL);
     S.bar = reinterpret_cast<uint64_t*>(S.cand + 64);
-    S.q = reinterpret_cast<float4*>(S.bar + 2);
+    S.q = reinterpret_cast<float4*>(S.bar + 4);
     S.stage = reinterpret_cast<float4*>(reinterpret_cast<float*>(S.q) + A.q_len);
     S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(S.stage) + STAGE_BYTES);
     if (lane == 0) {
         mbar_init(S.bar, 1u);
-        reinterpret_cast<uint32_t*>(S.bar + 1)[0] = 0u;   // phase parity
-        reinterpret_cast<uint32_t*>(S.bar + 1)[1] = 0u;   // copy-timeout flag
+        mbar_init(S.bar + 1, 1u);
+        reinterpret_cast<uint32_t*>(S.bar + 2)[0] = 0u;   // phase parities (bit 0, bit 1)
+        reinterpret_cast<uint32_t*>(S.bar + 2)[1] = 0u;   // copy-timeout flag
     }
     __syncwarp();
     uint32_t* bitmap = BITMAP ? A.bitmap + (size_t)(blockIdx.x * WARPS_PER_CTA + warp) * A.bitmap_words : nullptr;
@@ -210,7 +215,7 @@ frog_search_kernel(const FrogSearchArgs A) {
         int enc_hot_bytes = 0;                    // bytes of the first two chunks of a vertex's hotspot
         int second_pos = NO_POS;                  // pool position of the next unexpanded entry after `first`
         auto EVAL = [&](int ns_, uint32_t flag_, int off_ = 0, bool last_ = true) {
-            int f_ = evaluate_and_merge<EPL, F16, ROWB>(A.rows, A.row_bytes, A.slot_bytes, A.rows_per_pass, A.ef_s, S.pool,
+            int f_ = evaluate_and_merge<EPL, F16, ROWB, FROG_UNIQUE_MERGE && BITMAP>(A.rows, A.row_bytes, A.slot_bytes, A.rows_per_pass, A.ef_s, S.pool,
                                                   S.cand + off_, S.bar, S.q, S.stage, ns_, flag_, !BITMAP,
                                                   last_ ? enc_hot_base : nullptr,
                                                   (size_t)A.H * A.m, enc_hot_bytes, second_pos,
@@ -426,7 +431,7 @@ frog_search_kernel(const FrogSearchArgs A) {
         got = __reduce_add_sync(FULL, got);
         if (got < A.k) st |= FROG_ST_SHORT;
         if (__any_sync(FULL, forgets != 0)) st |= FROG_ST_FORGOT;   // counted per lane
-        if (reinterpret_cast<uint32_t*>(S.bar + 1)[1]) st |= FROG_ST_COPY_TIMEOUT;
+        if (reinterpret_cast<uint32_t*>(S.bar + 2)[1]) st |= FROG_ST_COPY_TIMEOUT;
         FROG_PHASE(4);
         if (lane == 0) {
             if (A.status) A.status[q] = st;
