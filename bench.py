@@ -35,10 +35,9 @@ SWEEP = [16, 24, 32, 40, 44, 48, 52, 56, 64, 80, 96, 112, 128, 160, 192, 256, 38
 BUDGETS = [16, 32, 48, 64]  # expansion budget B of Alg. 2: the paper's default up to the kernel's maximum
 RECALL_TARGET = 0.95
 HBM_FALLBACK_GBS = 6650.0
-# DRAM bytes of one search-kernel launch at the default bench point and its neighbours (sift 1M),
-# from the ncu captures summarised in profiles/frog_search_kernel_sift1m_b64_ef44.md
-NCU_TRAFFIC = {("sift", 1_000_000, 32, 112): 6.653e9, ("sift", 1_000_000, 64, 44): 5.187e9,
-               ("sift", 1_000_000, 64, 48): 5.514e9}
+# DRAM bytes of one search-kernel launch at the default bench point (sift 1M, B = 64, ef_s = 44),
+# from the ncu capture summarised in profiles/frog_search_kernel_sift1m_b64_ef44.md
+NCU_TRAFFIC = {("sift", 1_000_000, 64, 44): 5.174e9}
 
 
 def log(*a):
