@@ -312,87 +312,14 @@ __device__ __forceinline__ float staged_dist2(const float* __restrict__ vectors,
     return out;
 }
 
-// The same gather + distance with a run-time stage geometry and optional half-precision storage.
-// `rows` points at row-major data of `row_bytes` per row (fp32, or fp16 when F16); a row occupies a
-// slot of `slot_bytes` (>= the chunk, at most STAGE_CHUNK) in the stage buffer and up to
-// `rows_per_pass` (<= 16, multiple of 4) rows complete on one mbarrier phase.  fp16 elements are
-// converted to fp32 on the way out of shared memory; products and sums are fp32 in the same fixed
-// order, so the result equals the fp32 routine run on the rounded values bit for bit.
-// ROWB > 0 fixes the row size (and with it slot size and rows per pass) at compile time, which
-// unrolls the inner loops for the common shapes; ROWB == 0 takes the geometry from the arguments.
-template <bool F16, int ROWB = 0>
-__device__ __forceinline__ float staged_dist2_flex(const void* __restrict__ rows, int row_bytes, int slot_bytes,
-                                                   int rows_per_pass, const float4* qs, float4* stage, uint64_t* bar,
-                                                   uint32_t& phase, bool& ok, uint32_t my_rank, int ns, int lane) {
-    if (ROWB > 0) {
-        row_bytes = ROWB;
-        slot_bytes = ROWB >= STAGE_CHUNK ? STAGE_CHUNK : ROWB;     // ROWB is a power of two when below 512
-        rows_per_pass = (FROG_STAGE_ROWS * STAGE_CHUNK / slot_bytes) > 16 ? 16 : (FROG_STAGE_ROWS * STAGE_CHUNK / slot_bytes);
-    }
-    const int team = lane >> 3, sub = lane & 7;
-    constexpr int GROUP_BYTES = F16 ? 8 : 16;             // 4 elements
-    float out = 0.f;
-#pragma unroll 1
-    for (int r0 = 0; r0 < ns; r0 += rows_per_pass) {
-        const int nrows = min(rows_per_pass, ns - r0);
-        const int src = ((lane - r0) & 3) << 3;             // team that summed this lane's row
-        const uint32_t copy_rank = __shfl_sync(FULL, my_rank, (r0 + lane) & 31);
-        const char* src_row = reinterpret_cast<const char*>(rows) + (size_t)copy_rank * (size_t)row_bytes;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-        for (int c0 = 0; c0 < row_bytes; c0 += STAGE_CHUNK) {
-            const int cbytes = min(STAGE_CHUNK, row_bytes - c0);
-            __syncwarp();                                   // every lane is done reading the stage buffer
-            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(nrows * cbytes));
-            __syncwarp();
-            if (lane < nrows)
-                tma_load_1d(reinterpret_cast<char*>(stage) + lane * slot_bytes, src_row + c0, (uint32_t)cbytes, bar);
-            ok = mbar_wait(bar, phase) && ok;
-            phase ^= 1u;
-            const int g_lo = c0 / GROUP_BYTES, g_n = cbytes / GROUP_BYTES;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int r = i * 4 + team;
-                if (i * 4 < nrows && r < nrows) {
-                    const char* xrow = reinterpret_cast<const char*>(stage) + r * slot_bytes;
-#pragma unroll 4
-                    for (int g = sub; g < g_n; g += 8) {
-                        float4 x;
-                        if (F16) {
-                            const uint2 raw = *reinterpret_cast<const uint2*>(xrow + g * 8);
-                            const float2 lo2 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
-                            const float2 hi2 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
-                            x = make_float4(lo2.x, lo2.y, hi2.x, hi2.y);
-                        } else {
-                            x = *reinterpret_cast<const float4*>(xrow + g * 16);
-                        }
-                        const float4 q = qs[g_lo + g];
-                        float t;
-                        t = x.x - q.x; acc[i] = fmaf(t, t, acc[i]);
-                        t = x.y - q.y; acc[i] = fmaf(t, t, acc[i]);
-                        t = x.z - q.z; acc[i] = fmaf(t, t, acc[i]);
-                        t = x.w - q.w; acc[i] = fmaf(t, t, acc[i]);
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (i * 4 < nrows) {
-                float a = acc[i];
-                a = a + __shfl_xor_sync(FULL, a, 4);
-                a = a + __shfl_xor_sync(FULL, a, 2);
-                a = a + __shfl_xor_sync(FULL, a, 1);
-                const float v = __shfl_sync(FULL, a, src);
-                if (lane >= r0 && ((lane - r0) >> 2) == i && lane - r0 < nrows) out = v;
-            }
-        }
-    }
-    return out;
-}
-
-// The same computation as staged_dist2_flex with the stage buffer split into two halves, each with
-// its own mbarrier: while the teams reduce the rows of one half, the copies of the next group of
+// The same gather + distance for the search kernel, with a run-time row geometry and optional
+// half-precision storage.  `rows` points at row-major data of `row_bytes` per row (fp32, or fp16
+// when F16); a row, or its STAGE_CHUNK-byte column chunk, occupies a slot of `slot_bytes`.  fp16
+// elements are converted to fp32 on the way out of shared memory; products and sums are fp32 in
+// the same fixed order, so the result equals the fp32 routine run on the rounded values bit for
+// bit.  ROWB > 0 fixes the row size at compile time, which unrolls the inner loops for the common
+// shape; ROWB == 0 takes the geometry from the arguments.
+// The stage buffer is split into two halves, each with its own mbarrier: while the teams reduce the rows of one half, the copies of the next group of
 // rows are already landing in the other, so the arithmetic hides behind the copy latency.  A
 // group is up to 8 rows (4 for 512-byte slots: one row per team); a row longer than STAGE_CHUNK is
 // taken in column chunks, one chunk of every row of the group per step.  bar[0], bar[1] are the
@@ -403,11 +330,12 @@ __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows
                                                    uint32_t& phases, bool& ok, uint32_t my_rank, int ns, int lane) {
     if (ROWB > 0) {
         row_bytes = ROWB;
-        slot_bytes = ROWB >= STAGE_CHUNK ? STAGE_CHUNK : ROWB;     // ROWB is a power of two when below 512
+        slot_bytes = ROWB >= STAGE_CHUNK ? STAGE_CHUNK : ROWB;
     }
     constexpr int HALF = FROG_STAGE_ROWS * STAGE_CHUNK / 2;
     constexpr int GROUP_BYTES = F16 ? 8 : 16;             // 4 elements
-    const int rph = (HALF / slot_bytes) > 8 ? 8 : (HALF / slot_bytes);     // rows per half
+    constexpr int UNROLL_G = ROWB > 0 ? 4 : 1;            // the run-time geometry is short of registers
+    const int rph = (HALF / slot_bytes) >= 8 ? 8 : 4;     // rows per half: two rows or one row per team
     const int chunks = (row_bytes + STAGE_CHUNK - 1) / STAGE_CHUNK;
     const int steps = ((ns + rph - 1) / rph) * chunks;
     const int team = lane >> 3, sub = lane & 7;
@@ -444,7 +372,7 @@ __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows
             if ((i == 0 || rph > 4) && r < nrows) {
                 const char* xrow = half + r * slot_bytes;
                 float a = i == 0 ? acc0 : acc1;
-#pragma unroll 4
+#pragma unroll UNROLL_G
                 for (int gg = sub; gg < g_n; gg += 8) {
                     float4 x;
                     if (F16) {
@@ -490,18 +418,9 @@ __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows
     return out;
 }
 
-// two smallest values seen by a lane
-__device__ __forceinline__ void track2(int& m1, int& m2, int p) {
-    if (p < m1) { m2 = m1; m1 = p; }
-    else if (p < m2) m2 = p;
-}
-// warp-wide smallest and second smallest of the per-lane pairs (m1 <= m2), packed as
-// first | second << 16 (0xFFFF = none)
-__device__ __forceinline__ uint32_t first_two(int m1, int m2) {
-    const unsigned a = min((unsigned)m1, 0xFFFFu), b = min((unsigned)m2, 0xFFFFu);
-    const unsigned f = __reduce_min_sync(FULL, a);
-    const unsigned s2 = __reduce_min_sync(FULL, a == f ? b : a);
-    return f | (s2 << 16);
+// warp-wide smallest of the per-lane positions (0xFFFF = none)
+__device__ __forceinline__ uint32_t first_pos(int m1) {
+    return __reduce_min_sync(FULL, min((unsigned)m1, 0xFFFFu));
 }
 
 // Alg. 2 lines 15-17 in one pass.  `pool` holds ef_s (<= 32*EPL) keys ascending by key | 1,
@@ -510,8 +429,8 @@ __device__ __forceinline__ uint32_t first_two(int m1, int m2) {
 // index + (#new keys below it); everything landing at >= ef_s is dropped.  All counts come from
 // register compares and ballots: the new keys are broadcast one by one with shuffles, the lanes
 // hold the pool keys (lane l owns positions l, l+32, ...).  A new key equal to a pool key (a vertex
-// the visited table forgot) or to an earlier new key is discarded.  Returns the positions of the
-// first and of the second entry whose flag is 0, packed as first | second << 16 (0xFFFF = none).
+// the visited table forgot) or to an earlier new key is discarded.  Returns the position of the
+// first entry whose flag is 0 (0xFFFF = none).
 template <int EPL, bool UNIQUE = false>
 __device__ __forceinline__ uint32_t merge_batch(uint64_t* pool, uint64_t my_key, int ef_s, int lane) {
     uint64_t pk[EPL];
@@ -521,12 +440,12 @@ __device__ __forceinline__ uint32_t merge_batch(uint64_t* pool, uint64_t my_key,
     const uint64_t worst = pool[ef_s - 1];
     if ((my_key | 1ull) >= (worst | 1ull)) my_key = KEY_EMPTY;
     uint32_t have = __ballot_sync(FULL, my_key != KEY_EMPTY);
-    int m1 = NO_POS, m2 = NO_POS;
+    int m1 = NO_POS;
     if (have == 0) {
 #pragma unroll
         for (int e = 0; e < EPL; ++e)
-            if (pk[e] != KEY_EMPTY && !(pk[e] & 1ull)) track2(m1, m2, lane + 32 * e);
-        return first_two(m1, m2);
+            if (pk[e] != KEY_EMPTY && !(pk[e] & 1ull)) m1 = min(m1, lane + 32 * e);
+        return first_pos(m1);
     }
     int add[EPL];
 #pragma unroll
@@ -567,7 +486,7 @@ __device__ __forceinline__ uint32_t merge_batch(uint64_t* pool, uint64_t my_key,
             const int p = lane + 32 * e + add[e];
             if (p < ef_s) {
                 if (add[e]) pool[p] = pk[e];
-                if (!(pk[e] & 1ull)) track2(m1, m2, p);
+                if (!(pk[e] & 1ull)) m1 = min(m1, p);
             }
         }
     }
@@ -575,11 +494,11 @@ __device__ __forceinline__ uint32_t merge_batch(uint64_t* pool, uint64_t my_key,
         const int p = (32 * EPL - above) + rnew;
         if (p < ef_s) {
             pool[p] = my_key;
-            if (!(my_key & 1ull)) track2(m1, m2, p);
+            if (!(my_key & 1ull)) m1 = min(m1, p);
         }
     }
     __syncwarp();
-    return first_two(m1, m2);
+    return first_pos(m1);
 }
 
 // smallest key of the warp under the order key | 1 (KEY_EMPTY if no lane has one)

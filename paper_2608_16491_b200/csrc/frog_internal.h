@@ -50,8 +50,7 @@ struct FrogSearchArgs {
     const int32_t* order;      // processing order (heaviest first), or null: input order
     const void* rows;          // gather source: fp32 vectors, or their fp16 copy
     int row_bytes;             // bytes per stored row
-    int slot_bytes;            // bytes of one row slot in the stage buffer (power of two, <= 512)
-    int rows_per_pass;         // rows completing on one mbarrier phase (4..16)
+    int slot_bytes;            // bytes of one row slot in the stage buffer (multiple of 16, <= 512)
     int q_len;                 // floats of the query held in shared memory (8 * ceil(d / 8))
 };
 

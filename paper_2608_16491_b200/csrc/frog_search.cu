@@ -46,12 +46,6 @@ constexpr int WARPS_PER_CTA = FROG_WARPS_PER_CTA;
 #endif
 constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2, MODE_EAGER = 3;   // EAGER: FAST with the eager hash check
 
-#ifndef FROG_ENC_PREFETCH
-#define FROG_ENC_PREFETCH 1   // 0: off, 1: prefetch the predicted vertex's ENC lines
-#endif
-#ifndef FROG_PREFETCH_FN
-#define FROG_PREFETCH_FN prefetch_l2
-#endif
 #ifndef FROG_ENC_LD
 #define FROG_ENC_LD ldg_stream_u32
 #endif
@@ -104,12 +98,10 @@ __device__ __forceinline__ bool visited_test_and_set(const WarpSmem& S, uint32_t
 // three places of the kernel and inlining every copy costs registers and instruction cache.
 template <int EPL, bool F16, int ROWB, bool UNIQUE>
 __device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows, int row_bytes, int slot_bytes,
-                                                   int rows_per_pass, int ef_s,
+                                                   int ef_s,
                                                    uint64_t* pool, const uint32_t* cand, uint64_t* bar,
                                                    const float4* qs, float4* stage,
-                                                   int ns, uint32_t new_flag, bool dedupe,
-                                                   const uint32_t* enc_hot, size_t enc_stride, int enc_bytes,
-                                                   int next_pos, long long* t_dist) {
+                                                   int ns, uint32_t new_flag, bool dedupe, long long* t_dist) {
     const int lane = lane_id();
     uint32_t id = (lane < ns) ? cand[lane] : 0u;
     if (dedupe) {
@@ -141,23 +133,6 @@ __device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows
     }
     const uint64_t key = (lane < ns) ? make_key(d2, id, new_flag) : KEY_EMPTY;
     if (t_dist) *t_dist = clock64();
-#if FROG_ENC_PREFETCH
-    if (enc_hot) {
-        // The vertex expanded next is the smaller of the best new key that enters the pool and the
-        // pool's next unexpanded entry: start fetching the first lines of its ENC rows now, so the
-        // fetch overlaps the merge.  A wrong guess only wastes the prefetch.
-        uint64_t guess = warp_min_key(key);
-        const uint64_t worst = pool[ef_s - 1];
-        if ((guess | 1ull) >= (worst | 1ull)) guess = KEY_EMPTY;
-        const uint64_t nxt = next_pos < ef_s ? pool[next_pos] : KEY_EMPTY;
-        if ((nxt | 1ull) < (guess | 1ull)) guess = nxt;
-        if (guess != KEY_EMPTY) {
-            const char* p0 = reinterpret_cast<const char*>(enc_hot + (size_t)key_rank(guess) * enc_stride);
-            const char* line = reinterpret_cast<const char*>(reinterpret_cast<uintptr_t>(p0) & ~(uintptr_t)127) + 128 * lane;
-            if (lane < 3 && line < p0 + enc_bytes) FROG_PREFETCH_FN(line);
-        }
-    }
-#endif
     return (int)merge_batch<EPL, UNIQUE>(pool, key, ef_s, lane);
 }
 
@@ -211,14 +186,9 @@ frog_search_kernel(const FrogSearchArgs A) {
 
         // distance + merge call; in profile builds the time is split at the end of the distances
         long long t_split = 0;
-        const uint32_t* enc_hot_base = nullptr;   // ENC rows from L_start on (set once the hotspot is known)
-        int enc_hot_bytes = 0;                    // bytes of the first two chunks of a vertex's hotspot
-        int second_pos = NO_POS;                  // pool position of the next unexpanded entry after `first`
-        auto EVAL = [&](int ns_, uint32_t flag_, int off_ = 0, bool last_ = true) {
-            int f_ = evaluate_and_merge<EPL, F16, ROWB, FROG_UNIQUE_MERGE && BITMAP>(A.rows, A.row_bytes, A.slot_bytes, A.rows_per_pass, A.ef_s, S.pool,
+        auto EVAL = [&](int ns_, uint32_t flag_, int off_ = 0) {
+            int f_ = evaluate_and_merge<EPL, F16, ROWB, FROG_UNIQUE_MERGE && BITMAP>(A.rows, A.row_bytes, A.slot_bytes, A.ef_s, S.pool,
                                                   S.cand + off_, S.bar, S.q, S.stage, ns_, flag_, !BITMAP,
-                                                  last_ ? enc_hot_base : nullptr,
-                                                  (size_t)A.H * A.m, enc_hot_bytes, second_pos,
                                                   MODE == MODE_PROFILE ? &t_split : nullptr);
             if (MODE == MODE_PROFILE) {
                 long long n_ = clock64();
@@ -294,11 +264,7 @@ frog_search_kernel(const FrogSearchArgs A) {
             }
             FROG_PHASE(0);
             n_dist += ns;
-            enc_hot_base = A.enc + (size_t)L_start * A.m;
-            enc_hot_bytes = min(total, 64) * 4;
-            int packed = EVAL(ns, 0u);
-            int first = packed & 0xFFFF;
-            second_pos = (packed >> 16) & 0xFFFF;
+            int first = EVAL(ns, 0u);
             // lines 7-17
             while (first < A.ef_s) {
                 if ((int)n_exp >= A.max_iters) { st |= FROG_ST_ITER_CAP; break; }
@@ -403,13 +369,11 @@ frog_search_kernel(const FrogSearchArgs A) {
                 // lines 14-17; a budget above 32 can leave up to 64 survivors: two batches, the pool
                 // after both is the same as after one merge of all of them
                 if (ns > 32) {
-                    second_pos = EVAL(32, 0u, 0, false) & 0xFFFF;   // the next unexpanded entry so far
-                    packed = EVAL(ns - 32, 0u, 32);
+                    EVAL(32, 0u);
+                    first = EVAL(ns - 32, 0u, 32);
                 } else {
-                    packed = EVAL(ns, 0u);
+                    first = EVAL(ns, 0u);
                 }
-                first = packed & 0xFFFF;
-                second_pos = (packed >> 16) & 0xFFFF;
             }
         }
 
@@ -500,6 +464,15 @@ kernel_fn pick_kernel(int ef_s, int* pool_slots) {
     return frog_search_kernel<16, MODE, BITMAP, F16>;
 }
 
+template <int ROWB>
+kernel_fn pick_rowb(int ef_s) {
+    if (ef_s <= 32) return frog_search_kernel<1, MODE_FAST, true, false, ROWB>;
+    if (ef_s <= 64) return frog_search_kernel<2, MODE_FAST, true, false, ROWB>;
+    if (ef_s <= 128) return frog_search_kernel<4, MODE_FAST, true, false, ROWB>;
+    if (ef_s <= 256) return frog_search_kernel<8, MODE_FAST, true, false, ROWB>;
+    return frog_search_kernel<16, MODE_FAST, true, false, ROWB>;
+}
+
 struct LaunchPlan {
     kernel_fn fn;
     int grid, block, ctas_per_sm;
@@ -528,13 +501,13 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
         if (!bitmap || f16 || mode != MODE_FAST) return FROG_ERR_UNSUPPORTED;
         fn = pick_kernel<MODE_EAGER, true, false>(beam_width, &pool_slots);
     }
-    // common shape with the geometry fixed at compile time: fp32 rows of 512 bytes (d = 125..128)
-    if (mode == MODE_FAST && bitmap && !f16 && !P.eager_hash && ix->info.d_pad == 128) {
-        if (beam_width <= 32) fn = frog_search_kernel<1, MODE_FAST, true, false, 512>;
-        else if (beam_width <= 64) fn = frog_search_kernel<2, MODE_FAST, true, false, 512>;
-        else if (beam_width <= 128) fn = frog_search_kernel<4, MODE_FAST, true, false, 512>;
-        else if (beam_width <= 256) fn = frog_search_kernel<8, MODE_FAST, true, false, 512>;
-        else fn = frog_search_kernel<16, MODE_FAST, true, false, 512>;
+    // common shapes with the row geometry fixed at compile time (fp32 rows of 384, 512 and 3072 bytes:
+    // d = 96, 128, 768)
+    if (mode == MODE_FAST && bitmap && !f16 && !P.eager_hash) {
+        const int rb = ix->info.d_pad * 4;
+        if (rb == 512) fn = pick_rowb<512>(beam_width);
+        else if (rb == 384) fn = pick_rowb<384>(beam_width);
+        else if (rb == 3072) fn = pick_rowb<3072>(beam_width);
     }
     size_t smem = warp_smem_bytes(pool_slots, query_len(ix->info.d), P.hash_bits, bitmap) * WARPS_PER_CTA;
     if (smem > 227 * 1024) return FROG_ERR_UNSUPPORTED;
@@ -558,18 +531,12 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
     return FROG_OK;
 }
 
-// gather source and stage geometry: a row slot is the row (or its 512-byte chunk) rounded up to a
-// power of two; as many rows as fit the stage buffer (at most 16, a multiple of 4) share one phase
+// gather source and stage geometry: a row slot is the row, or its 512-byte chunk
 void set_gather(const frog_index* ix, bool f16, FrogSearchArgs* A) {
     const int d_pad_h = query_len(ix->info.d);
     A->rows = f16 ? ix->d_vectors_h : (const void*)ix->d_vectors;
     A->row_bytes = f16 ? d_pad_h * 2 : ix->info.d_pad * 4;
-    int slot = 16;
-    while (slot < A->row_bytes && slot < STAGE_CHUNK) slot <<= 1;
-    A->slot_bytes = slot;
-    int rows = STAGE_BYTES / slot;
-    rows = rows > 16 ? 16 : rows;
-    A->rows_per_pass = rows;
+    A->slot_bytes = A->row_bytes < STAGE_CHUNK ? A->row_bytes : STAGE_CHUNK;   // rows are 16-byte multiples
     A->q_len = d_pad_h;
 }
 
