@@ -509,11 +509,4 @@ __device__ __forceinline__ uint64_t warp_min_key(uint64_t key) {
     return ((uint64_t)mhi << 32) | mlo;
 }
 
-__device__ __forceinline__ void prefetch_l1(const void* p) {
-    asm volatile("prefetch.global.L1 [%0];" ::"l"(p));
-}
-__device__ __forceinline__ void prefetch_l2(const void* p) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
-}
-
 }  // namespace frogdev
