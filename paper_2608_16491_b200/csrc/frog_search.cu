@@ -31,24 +31,12 @@ constexpr int WARPS_PER_CTA = FROG_WARPS_PER_CTA;
 #ifndef FROG_MINB
 #define FROG_MINB 16          // resident CTAs per SM the register allocation aims at (EPL <= 4)
 #endif
-#ifndef FROG_NG
-#define FROG_NG 2
-#endif
 
 #ifndef FROG_MINB_BIG
 #define FROG_MINB_BIG 4       // the same for pools above 128 entries
 #endif
-#ifndef FROG_UNIQUE_MERGE
-#define FROG_UNIQUE_MERGE 1   // bitmap visited set: keys reaching the merge are distinct, skip the copy test
-#endif
-#ifndef FROG_EVAL_INLINE
-#define FROG_EVAL_INLINE __noinline__
-#endif
 constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2, MODE_EAGER = 3;   // EAGER: FAST with the eager hash check
 
-#ifndef FROG_ENC_LD
-#define FROG_ENC_LD ldg_stream_u32
-#endif
 constexpr int STAGE_BYTES = FROG_STAGE_ROWS * STAGE_CHUNK;
 
 // per-warp shared memory: pool | candidate list | two mbarriers, their parities, a failure flag | query | stage | hash
@@ -97,7 +85,7 @@ __device__ __forceinline__ bool visited_test_and_set(const WarpSmem& S, uint32_t
 // lines 14-17).  Returns the first unexpanded pool position.  Kept out of line: it is called from
 // three places of the kernel and inlining every copy costs registers and instruction cache.
 template <int EPL, bool F16, int ROWB, bool UNIQUE>
-__device__ FROG_EVAL_INLINE int evaluate_and_merge(const void* __restrict__ rows, int row_bytes, int slot_bytes,
+__device__ __noinline__ int evaluate_and_merge(const void* __restrict__ rows, int row_bytes, int slot_bytes,
                                                    int ef_s,
                                                    uint64_t* pool, const uint32_t* cand, uint64_t* bar,
                                                    const float4* qs, float4* stage,
@@ -187,7 +175,7 @@ frog_search_kernel(const FrogSearchArgs A) {
         // distance + merge call; in profile builds the time is split at the end of the distances
         long long t_split = 0;
         auto EVAL = [&](int ns_, uint32_t flag_, int off_ = 0) {
-            int f_ = evaluate_and_merge<EPL, F16, ROWB, FROG_UNIQUE_MERGE && BITMAP>(A.rows, A.row_bytes, A.slot_bytes, A.ef_s, S.pool,
+            int f_ = evaluate_and_merge<EPL, F16, ROWB, BITMAP>(A.rows, A.row_bytes, A.slot_bytes, A.ef_s, S.pool,
                                                   S.cand + off_, S.bar, S.q, S.stage, ns_, flag_, !BITMAP,
                                                   MODE == MODE_PROFILE ? &t_split : nullptr);
             if (MODE == MODE_PROFILE) {
@@ -289,7 +277,7 @@ frog_search_kernel(const FrogSearchArgs A) {
                     // admitted, finds the bit set and is dropped).
                     for (int c0 = 0; c0 < total && cnt < A.B; c0 += 32) {
                         uint32_t v = BOT;
-                        if (c0 + lane < total) v = FROG_ENC_LD(hot + c0 + lane);
+                        if (c0 + lane < total) v = ldg_stream_u32(hot + c0 + lane);
                         const bool in_range = (v - (uint32_t)l_q) <= span;
                         const uint32_t bit = 1u << (v & 31);
                         uint32_t word = 0xFFFFFFFFu;
@@ -310,8 +298,8 @@ frog_search_kernel(const FrogSearchArgs A) {
                 } else
                 for (int c0 = 0; c0 < total && cnt < A.B; c0 += 64) {
                     uint32_t v0 = BOT, v1 = BOT;
-                    if (c0 + lane < total) v0 = FROG_ENC_LD(hot + c0 + lane);
-                    if (c0 + 32 + lane < total) v1 = FROG_ENC_LD(hot + c0 + 32 + lane);
+                    if (c0 + lane < total) v0 = ldg_stream_u32(hot + c0 + lane);
+                    if (c0 + 32 + lane < total) v1 = ldg_stream_u32(hot + c0 + 32 + lane);
                     // first chunk
                     const bool pred0 = (v0 - (uint32_t)l_q) <= span;
                     const uint32_t M0 = __ballot_sync(FULL, pred0);
@@ -515,9 +503,6 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
     int per_sm = 0;
     FROG_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)fn, WARPS_PER_CTA * 32, smem));
     if (per_sm < 1) return FROG_ERR_UNSUPPORTED;
-#ifdef FROG_CAP_CTAS
-    if (per_sm > FROG_CAP_CTAS) per_sm = FROG_CAP_CTAS;
-#endif
     int grid = per_sm * ix->sm_count;
     if (nq > 0) {
         int need = (nq + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
