@@ -32,8 +32,11 @@ constexpr int WARPS_PER_CTA = FROG_WARPS_PER_CTA;
 #define FROG_MINB 16          // resident CTAs per SM the register allocation aims at (EPL <= 4)
 #endif
 
-#ifndef FROG_MINB_BIG
-#define FROG_MINB_BIG 4       // the same for pools above 128 entries
+#ifndef FROG_MINB_8
+#define FROG_MINB_8 12        // the same for pools of 256 entries (80 registers)
+#endif
+#ifndef FROG_MINB_16
+#define FROG_MINB_16 10       // and of 512 entries (96 registers)
 #endif
 constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2, MODE_EAGER = 3;   // EAGER: FAST with the eager hash check
 
@@ -83,16 +86,16 @@ __device__ __forceinline__ bool visited_test_and_set(const WarpSmem& S, uint32_t
 
 // Distances of the ns <= 32 ranks listed in cand[0..ns) and their merge into the pool (Alg. 2
 // lines 14-17).  Returns the first unexpanded pool position.  Kept out of line: it is called from
-// three places of the kernel and inlining every copy costs registers and instruction cache.
+// several places of the kernel and inlining every copy costs registers and instruction cache.
+// UNIQUE: the visited set is exact (bitmap form), so the ranks are distinct and none is in the pool.
 template <int EPL, bool F16, int ROWB, bool UNIQUE>
-__device__ __noinline__ int evaluate_and_merge(const void* __restrict__ rows, int row_bytes, int slot_bytes,
-                                                   int ef_s,
-                                                   uint64_t* pool, const uint32_t* cand, uint64_t* bar,
-                                                   const float4* qs, float4* stage,
-                                                   int ns, uint32_t new_flag, bool dedupe, long long* t_dist) {
+__device__ __noinline__ int evaluate_and_merge(const void* __restrict__ rows, int row_bytes, int slot_bytes, int ef_s,
+                                               uint64_t* pool, const uint32_t* cand, uint64_t* bar,
+                                               const float4* qs, float4* stage, int ns, uint32_t new_flag,
+                                               long long* t_dist) {
     const int lane = lane_id();
     uint32_t id = (lane < ns) ? cand[lane] : 0u;
-    if (dedupe) {
+    if (!UNIQUE) {
         // The shared-memory visited table can let the same rank through twice in one batch once it
         // starts dropping entries.  Two bulk copies of one source row completing on the same
         // mbarrier were observed to leave the barrier incomplete (the wait ran into its polling
@@ -126,7 +129,7 @@ __device__ __noinline__ int evaluate_and_merge(const void* __restrict__ rows, in
 
 template <int EPL, int MODE, bool BITMAP, bool F16, int ROWB = 0>
 __global__ void __launch_bounds__(WARPS_PER_CTA * 32,
-                                  (MODE == MODE_FAST || MODE == MODE_EAGER) ? (EPL <= 4 ? FROG_MINB : FROG_MINB_BIG) : 1)
+                                  (MODE == MODE_FAST || MODE == MODE_EAGER) ? (EPL <= 4 ? FROG_MINB : EPL == 8 ? FROG_MINB_8 : FROG_MINB_16) : 1)
 frog_search_kernel(const FrogSearchArgs A) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int lane = lane_id();
@@ -176,7 +179,7 @@ frog_search_kernel(const FrogSearchArgs A) {
         long long t_split = 0;
         auto EVAL = [&](int ns_, uint32_t flag_, int off_ = 0) {
             int f_ = evaluate_and_merge<EPL, F16, ROWB, BITMAP>(A.rows, A.row_bytes, A.slot_bytes, A.ef_s, S.pool,
-                                                  S.cand + off_, S.bar, S.q, S.stage, ns_, flag_, !BITMAP,
+                                                  S.cand + off_, S.bar, S.q, S.stage, ns_, flag_,
                                                   MODE == MODE_PROFILE ? &t_split : nullptr);
             if (MODE == MODE_PROFILE) {
                 long long n_ = clock64();
