@@ -392,7 +392,9 @@ def run_ours(args):
                    "launch": launch, "sweep": sweep},
         "e2e": {"value": ws * nq * args.steps / e2e_s_max, "unit": UNIT,
                 "h2d_bytes_per_step": nq * info.d * 4 + 2 * nq * 4, "d2h_bytes_per_step": 2 * nq * k * 4,
-                "same_ids_as_device_path": e2e_same},
+                "same_ids_as_device_path": e2e_same,
+                "transfer": "pinned host buffers, read and written by the kernels across the bus inside the "
+                            "timed region (frog_search_host); wall clock per call including its stream sync"},
         "gpu_launches": 3 * args.steps,   # per step: endpoint/plan kernel, order kernel, search kernel
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src,

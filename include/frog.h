@@ -167,9 +167,11 @@ int frog_exact_search(const frog_index_t* index, const float* queries, const int
                       int nq, int k, int32_t* out_ids, float* out_dists, void* stream);
 
 /* frog_search_host: the end-to-end call of the paper's timing scope (Sec. 8.1.3: transfer of
- * query vectors and ranges, then execution).  All pointers are HOST memory (pinned memory makes
- * the copies asynchronous); copies in, searches, copies the results out and synchronises the
- * stream.  Uses staging buffers owned by the index, grown on first use. */
+ * query vectors and ranges, then execution).  All pointers are HOST memory.  If all five buffers
+ * are page-locked and device-mapped (cudaHostAlloc / cudaHostRegister) the kernels read the inputs
+ * and write the results across the bus themselves, overlapping the transfers with the search;
+ * otherwise the call copies in through staging buffers owned by the index (grown on first use),
+ * searches and copies the results out.  Either way it returns after synchronising the stream. */
 int frog_search_host(frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
                      int nq, int k, int beam_width, const frog_params_t* params /* HOST, may be null */,
                      int32_t* out_ids, float* out_dists, void* stream);

@@ -216,6 +216,29 @@ extern "C" int frog_search_host(frog_index_t* ix, const float* queries, const in
     if (!queries || !lo || !hi || !out_ids || !out_dists) return FROG_ERR_INVALID_ARG;
     FROG_CUDA_TRY(cudaSetDevice(ix->info.device));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // Pinned (page-locked, device-mapped) host buffers need no staging: the kernels read each query
+    // and write each result row across the bus themselves, so the transfers overlap the search
+    // instead of bracketing it.  Pageable buffers take the staged path below.
+    {
+        const void* host[5] = {queries, lo, hi, out_ids, out_dists};
+        void* dev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+        bool mapped = true;
+        for (int i = 0; i < 5 && mapped; ++i) {
+            cudaPointerAttributes at;
+            if (cudaPointerGetAttributes(&at, host[i]) != cudaSuccess) { cudaGetLastError(); mapped = false; break; }
+            mapped = at.type == cudaMemoryTypeHost && at.devicePointer != nullptr;
+            dev[i] = at.devicePointer;
+        }
+        if (mapped) {
+            int rc = frog_search_ex(ix, static_cast<const float*>(dev[0]), static_cast<const int32_t*>(dev[1]),
+                                    static_cast<const int32_t*>(dev[2]), nq, k, beam_width, params,
+                                    static_cast<int32_t*>(dev[3]), static_cast<float*>(dev[4]), nullptr, nullptr,
+                                    nullptr, 0, stream);
+            if (rc != FROG_OK) return rc;
+            FROG_CUDA_TRY(cudaStreamSynchronize(s));
+            return FROG_OK;
+        }
+    }
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
     const size_t b_q = up((size_t)nq * ix->info.d * 4), b_r = up((size_t)nq * 4), b_o = up((size_t)nq * k * 4);
     const size_t need = b_q + 2 * b_r + 2 * b_o;

@@ -227,7 +227,11 @@ def test_host_buffer_call_matches(libs, tiny_gpu):
                                  torch.from_numpy(wl.lo).pin_memory(),
                                  torch.from_numpy(wl.hi).pin_memory(), wl.k, 64)
     assert np.array_equal(ids.numpy(), ref.ids) and np.array_equal(dists.numpy(), ref.dists)
-    # a second, larger call regrows the staging area
+    # pageable inputs and outputs take the staged path; a second, larger call regrows the staging area
+    p_ids = torch.empty((wl.nq, wl.k), dtype=torch.int32)
+    p_d = torch.empty((wl.nq, wl.k), dtype=torch.float32)
+    gix.search_host(wl.queries, wl.lo, wl.hi, wl.k, 64, out_ids=p_ids, out_dists=p_d)
+    assert np.array_equal(p_ids.numpy(), ref.ids) and np.array_equal(p_d.numpy(), ref.dists)
     reps = 3
     Q = np.tile(wl.queries, (reps, 1))
     ids, dists = gix.search_host(Q, np.tile(wl.lo, reps), np.tile(wl.hi, reps), wl.k, 64)
