@@ -137,10 +137,14 @@ int frog_index_enable_f16(frog_index_t* index);
  *   out_dists  DEVICE, nq x k fp32: L2 distances (not squared), ascending; +inf padding
  *   stream     cudaStream_t (as void*); the call only enqueues work and returns
  * The caller owns all buffers and keeps them alive until the stream reaches the end of the
- * call.  Calls on the same index must not overlap on the GPU (they share the index's scratch:
- * a work counter and the visited slabs); serialise them on one stream or with events.  The
- * first call (and any call that needs more resident warps than all calls before it) allocates
- * the visited slabs with cudaMalloc after a device synchronise.  nq == 0 is a no-op.
+ * call.  One index may be searched from several streams and host threads at once: a launch
+ * borrows one of up to four scratch sets owned by the index (work counter, visited slabs,
+ * planning arrays); a stream keeps the set it used last, another stream gets an idle or a new
+ * set, and when all four are busy the stream is made to wait for the one unused the longest.
+ * Launches on different streams can therefore overlap on the GPU (the next batch fills the warps
+ * that the last queries of the previous one leave idle).  The first call on a stream (and any
+ * call that needs more resident warps than the calls before it) allocates visited slabs with
+ * cudaMalloc after a device synchronise.  nq == 0 is a no-op.
  * Errors: INVALID_ARG, UNSUPPORTED, CUDA (launch failure).  Per-query conditions (empty range,
  * iteration cap, fewer than k results) are not errors; see frog_search_ex. */
 int frog_search(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,

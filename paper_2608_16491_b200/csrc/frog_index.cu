@@ -48,13 +48,11 @@ int alloc_device(frog_index* ix) {
     if ((e = cudaMalloc(&ix->d_sorted_attr, b_attr)) != cudaSuccess ||
         (e = cudaMalloc(&ix->d_rank2id, b_attr)) != cudaSuccess ||
         (e = cudaMalloc(&ix->d_vectors, b_vec)) != cudaSuccess ||
-        (e = cudaMalloc(&ix->d_enc, b_enc)) != cudaSuccess ||
-        (e = cudaMalloc(&ix->d_work, 1024)) != cudaSuccess) {
+        (e = cudaMalloc(&ix->d_enc, b_enc)) != cudaSuccess) {
         froghost::set_cuda_error(e);
         return e == cudaErrorMemoryAllocation ? FROG_ERR_NOMEM : FROG_ERR_CUDA;
     }
-    ix->info.device_bytes = (int64_t)(2 * b_attr + b_vec + b_enc + 1024);
-    FROG_CUDA_TRY(cudaMemset(ix->d_work, 0, 1024));
+    ix->info.device_bytes = (int64_t)(2 * b_attr + b_vec + b_enc);
     cudaDeviceProp prop;
     FROG_CUDA_TRY(cudaGetDeviceProperties(&prop, I.device));
     ix->sm_count = prop.multiProcessorCount;
@@ -113,9 +111,12 @@ extern "C" void frog_index_free(frog_index_t* ix) {
         cudaFree(ix->d_vectors);
         cudaFree(ix->d_vectors_h);
         cudaFree(ix->d_enc);
-        cudaFree(ix->d_work);
-        cudaFree(ix->d_bitmap);
-        cudaFree(ix->d_plan);
+        for (int i = 0; i < ix->n_scratch; ++i) {
+            cudaFree(ix->scratch[i].d_work);
+            cudaFree(ix->scratch[i].d_bitmap);
+            cudaFree(ix->scratch[i].d_plan);
+            if (ix->scratch[i].done) cudaEventDestroy(ix->scratch[i].done);
+        }
         cudaFree(ix->d_stage);
     }
     delete ix;
@@ -239,6 +240,7 @@ extern "C" int frog_search_host(frog_index_t* ix, const float* queries, const in
             return FROG_OK;
         }
     }
+    std::lock_guard<std::mutex> stage_lock(ix->stage_mu);
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
     const size_t b_q = up((size_t)nq * ix->info.d * 4), b_r = up((size_t)nq * 4), b_o = up((size_t)nq * k * 4);
     const size_t need = b_q + 2 * b_r + 2 * b_o;

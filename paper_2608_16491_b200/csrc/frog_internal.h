@@ -2,9 +2,25 @@
 #pragma once
 
 #include <cstdint>
+#include <mutex>
 #include <cuda_runtime.h>
 
 #include "frog.h"
+
+// One set of search scratch: the work counter of the persistent kernel (+ planning histogram), the
+// per-warp visited slabs, the per-query planning arrays, and an event marking the end of the last
+// launch that used the set.
+struct FrogScratch {
+    unsigned int* d_work = nullptr;  // 1 KB
+    uint32_t* d_bitmap = nullptr;    // bitmap_slots x words per slot
+    size_t bitmap_slots = 0;
+    int32_t* d_plan = nullptr;       // per query: rank interval (2 ints) and processing order (1 int)
+    size_t plan_queries = 0;
+    cudaEvent_t done = nullptr;
+    cudaStream_t stream = nullptr;   // stream of the last launch
+    unsigned long long tick = 0;
+};
+constexpr int FROG_SCRATCH_SETS = 4;
 
 struct frog_index {
     frog_index_info_t info;
@@ -13,14 +29,16 @@ struct frog_index {
     float* d_vectors = nullptr;      // n x d_pad, rank order
     void* d_vectors_h = nullptr;     // optional fp16 copy, n x d_pad_h (d_pad_h = 8 * ceil(d / 8))
     uint32_t* d_enc = nullptr;       // n x H x m
-    unsigned int* d_work = nullptr;  // scratch: work counter of the persistent kernel (+ spare words)
-    uint32_t* d_bitmap = nullptr;    // scratch: per-warp visited slabs (bitmap_slots x words per slot)
-    size_t bitmap_slots = 0;
-    int32_t* d_plan = nullptr;       // scratch: per-query rank interval (2 ints) and processing order (1 int)
-    size_t plan_queries = 0;
+    // Scratch of the search launches.  A launch borrows one set; sets are handed out so that launches
+    // on different streams never share one while either may still be running (see acquire_scratch).
+    FrogScratch scratch[FROG_SCRATCH_SETS];
+    int n_scratch = 0;
+    unsigned long long tick = 0;     // launch counter, for least-recently-used selection
+    std::mutex mu;                   // guards the scratch sets and the order of launches into them
     // staging for frog_search_host, grown on demand
     void* d_stage = nullptr;
     size_t stage_bytes = 0;
+    std::mutex stage_mu;             // one staged host call at a time
     int sm_count = 0;
 };
 
@@ -57,8 +75,9 @@ struct FrogSearchArgs {
 namespace froghost {
 void set_cuda_error(cudaError_t e);
 int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in, frog_params_t* out);
-int ensure_bitmap(const frog_index* ix, size_t slots);
-int ensure_plan(const frog_index* ix, size_t nq);
+int acquire_scratch(frog_index* ix, cudaStream_t s, FrogScratch** out);
+int ensure_bitmap(const frog_index* ix, FrogScratch* sc, size_t slots);
+int ensure_plan(FrogScratch* sc, size_t nq);
 }  // namespace froghost
 
 #define FROG_CUDA_TRY(expr)                                  \

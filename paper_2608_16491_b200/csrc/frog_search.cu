@@ -565,41 +565,79 @@ int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in
     return FROG_OK;
 }
 
-// Make sure the index owns a visited slab for `slots` resident warps.  Grows (cudaFree + cudaMalloc,
+// Scratch set for a launch on stream s.  Launches of one stream are ordered by the stream, so a
+// stream keeps the set it used last.  Otherwise an idle set (its last launch has finished) is
+// taken, or a new one is created while fewer than FROG_SCRATCH_SETS exist, or the stream is made
+// to wait for the set that has been unused the longest.  Called with ix->mu held.
+int acquire_scratch(frog_index* ix, cudaStream_t s, FrogScratch** out) {
+    FrogScratch* pick = nullptr;
+    for (int i = 0; i < ix->n_scratch && !pick; ++i)
+        if (ix->scratch[i].tick && ix->scratch[i].stream == s) pick = &ix->scratch[i];
+    for (int i = 0; i < ix->n_scratch && !pick; ++i) {
+        FrogScratch& sc = ix->scratch[i];
+        if (!sc.tick) { pick = &sc; break; }
+        const cudaError_t q = cudaEventQuery(sc.done);
+        if (q == cudaSuccess) pick = &sc;
+        else if (q == cudaErrorNotReady) cudaGetLastError();
+        else { set_cuda_error(q); return FROG_ERR_CUDA; }
+    }
+    if (!pick && ix->n_scratch < FROG_SCRATCH_SETS) {
+        FrogScratch& sc = ix->scratch[ix->n_scratch];
+        cudaError_t e = cudaMalloc(&sc.d_work, 1024);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sc.done, cudaEventDisableTiming);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            if (sc.d_work) cudaFree(sc.d_work);
+            sc.d_work = nullptr;
+            if (ix->n_scratch == 0) { set_cuda_error(e); return e == cudaErrorMemoryAllocation ? FROG_ERR_NOMEM : FROG_ERR_CUDA; }
+        } else {
+            ++ix->n_scratch;
+            pick = &sc;
+        }
+    }
+    if (!pick) {
+        pick = &ix->scratch[0];
+        for (int i = 1; i < ix->n_scratch; ++i)
+            if (ix->scratch[i].tick < pick->tick) pick = &ix->scratch[i];
+        FROG_CUDA_TRY(cudaStreamWaitEvent(s, pick->done, 0));
+    }
+    *out = pick;
+    return FROG_OK;
+}
+
+// Make sure the set owns a visited slab for `slots` resident warps.  Grows (cudaFree + cudaMalloc,
 // after synchronising the device) only when a launch needs more slots than any launch before it.
-int ensure_bitmap(const frog_index* cix, size_t slots) {
-    frog_index* ix = const_cast<frog_index*>(cix);
+int ensure_bitmap(const frog_index* ix, FrogScratch* sc, size_t slots) {
     const size_t words = bitmap_words_per_slot(ix);
-    if (ix->d_bitmap && ix->bitmap_slots >= slots) return FROG_OK;
+    if (sc->d_bitmap && sc->bitmap_slots >= slots) return FROG_OK;
     FROG_CUDA_TRY(cudaDeviceSynchronize());
-    if (ix->d_bitmap) FROG_CUDA_TRY(cudaFree(ix->d_bitmap));
-    ix->d_bitmap = nullptr;
-    ix->bitmap_slots = 0;
-    cudaError_t e = cudaMalloc(&ix->d_bitmap, slots * words * sizeof(uint32_t));
+    if (sc->d_bitmap) FROG_CUDA_TRY(cudaFree(sc->d_bitmap));
+    sc->d_bitmap = nullptr;
+    sc->bitmap_slots = 0;
+    cudaError_t e = cudaMalloc(&sc->d_bitmap, slots * words * sizeof(uint32_t));
     if (e != cudaSuccess) {
         cudaGetLastError();
         set_cuda_error(e);
         return FROG_ERR_NOMEM;
     }
-    ix->bitmap_slots = slots;
+    sc->bitmap_slots = slots;
     return FROG_OK;
 }
 
 // Per-query planning scratch: 3 ints per query, grown when a batch is larger than any before.
-int ensure_plan(const frog_index* cix, size_t nq) {
-    frog_index* ix = const_cast<frog_index*>(cix);
-    if (ix->d_plan && ix->plan_queries >= nq) return FROG_OK;
+int ensure_plan(FrogScratch* sc, size_t nq) {
+    if (sc->d_plan && sc->plan_queries >= nq) return FROG_OK;
     FROG_CUDA_TRY(cudaDeviceSynchronize());
-    if (ix->d_plan) FROG_CUDA_TRY(cudaFree(ix->d_plan));
-    ix->d_plan = nullptr;
-    ix->plan_queries = 0;
-    cudaError_t e = cudaMalloc(&ix->d_plan, nq * 3 * sizeof(int32_t));
+    if (sc->d_plan) FROG_CUDA_TRY(cudaFree(sc->d_plan));
+    sc->d_plan = nullptr;
+    sc->plan_queries = 0;
+    cudaError_t e = cudaMalloc(&sc->d_plan, nq * 3 * sizeof(int32_t));
     if (e != cudaSuccess) {
         cudaGetLastError();
         set_cuda_error(e);
         return FROG_ERR_NOMEM;
     }
-    ix->plan_queries = nq;
+    sc->plan_queries = nq;
     return FROG_OK;
 }
 
@@ -640,8 +678,14 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     LaunchPlan plan;
     rc = plan_launch(index, beam_width, P, mode, bitmap, nq, &plan);
     if (rc) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    frog_index* mix = const_cast<frog_index*>(index);      // the scratch sets are the index's only mutable part
+    std::lock_guard<std::mutex> lock(mix->mu);
+    FrogScratch* sc = nullptr;
+    rc = froghost::acquire_scratch(mix, s, &sc);
+    if (rc) return rc;
     if (bitmap) {
-        rc = froghost::ensure_bitmap(index, (size_t)plan.grid * WARPS_PER_CTA);
+        rc = froghost::ensure_bitmap(index, sc, (size_t)plan.grid * WARPS_PER_CTA);
         if (rc == FROG_ERR_NOMEM && P.visited == FROG_VISITED_AUTO) {
             // no room for the slabs: fall back to the shared-memory table
             bitmap = false;
@@ -679,28 +723,29 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     A.stats = stats;
     A.trace = trace;
     A.trace_cap = trace_cap;
-    A.work_counter = index->d_work;
-    A.bitmap = bitmap ? index->d_bitmap : nullptr;
+    A.work_counter = sc->d_work;
+    A.bitmap = bitmap ? sc->d_bitmap : nullptr;
     A.bitmap_words = bitmap_words_per_slot(index);
     A.ranges = nullptr;
     A.order = nullptr;
     set_gather(index, P.storage == FROG_STORAGE_F16, &A);
 
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    FROG_CUDA_TRY(cudaMemsetAsync(index->d_work, 0, 1024, s));
+    FROG_CUDA_TRY(cudaMemsetAsync(sc->d_work, 0, 1024, s));
     // planning pass (skipped for tiny batches and when its scratch cannot be had)
-    const bool planned = !(P.debug_flags & 2) && nq >= 64 && froghost::ensure_plan(index, (size_t)nq) == FROG_OK;
+    const bool planned = !(P.debug_flags & 2) && nq >= 64 && froghost::ensure_plan(sc, (size_t)nq) == FROG_OK;
     if (planned) {
-        int2* ranges = reinterpret_cast<int2*>(index->d_plan);
-        int32_t* order = index->d_plan + 2 * (size_t)index->plan_queries;
-        frog_plan_kernel<<<(nq * 32 + 255) / 256, 256, 0, s>>>(index->d_sorted_attr, A.n, lo, hi, nq, ranges,
-                                                               index->d_work);
-        frog_order_kernel<<<(nq + 255) / 256, 256, 0, s>>>(lo, hi, nq, ranges, order, index->d_work);
+        int2* ranges = reinterpret_cast<int2*>(sc->d_plan);
+        int32_t* order = sc->d_plan + 2 * sc->plan_queries;
+        frog_plan_kernel<<<(nq * 32 + 255) / 256, 256, 0, s>>>(index->d_sorted_attr, A.n, lo, hi, nq, ranges, sc->d_work);
+        frog_order_kernel<<<(nq + 255) / 256, 256, 0, s>>>(lo, hi, nq, ranges, order, sc->d_work);
         A.ranges = ranges;
         A.order = order;
     }
     plan.fn<<<plan.grid, plan.block, plan.smem, s>>>(A);
     FROG_CUDA_TRY(cudaGetLastError());
+    FROG_CUDA_TRY(cudaEventRecord(sc->done, s));
+    sc->stream = s;
+    sc->tick = ++mix->tick;
     return FROG_OK;
 }
 

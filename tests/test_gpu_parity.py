@@ -152,6 +152,26 @@ def test_side_stream_and_back_to_back_calls(libs, tiny_gpu):
     assert np.array_equal(b_ids.cpu().numpy(), ref_b.ids) and np.array_equal(b_d.cpu().numpy(), ref_b.dists)
 
 
+def test_concurrent_streams_share_one_index(libs, tiny_gpu):
+    """Searches issued on different streams may overlap on the GPU: each stream works on its own
+    scratch set (work counter, visited slabs, planning arrays), so the answers are those of
+    separate calls.  More streams than scratch sets exist are served too (they queue)."""
+    wl, ix, gix = tiny_gpu
+    q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
+    cfgs = [(32, 64), (96, 16), (48, 32), (64, 64), (24, 8), (128, 16)]          # (beam, budget) per stream
+    refs = [oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, ef, B=B) for ef, B in cfgs]
+    streams = [torch.cuda.Stream() for _ in cfgs]
+    torch.cuda.synchronize()
+    outs = [[] for _ in cfgs]
+    for rep in range(4):
+        for j, (ef, B) in enumerate(cfgs):
+            outs[j].append(gix.search(q, lo, hi, wl.k, ef, stream=streams[j], params=libs.Params(budget=B)))
+    torch.cuda.synchronize()
+    for j, ref in enumerate(refs):
+        for ids, dists in outs[j]:
+            assert np.array_equal(ids.cpu().numpy(), ref.ids) and np.array_equal(dists.cpu().numpy(), ref.dists)
+
+
 def test_non_finite_queries_terminate(libs, tiny_gpu):
     """Non-finite query components: the results are unspecified, but the call returns, every
     reported id lies in the query's range and no wait ran into its limit."""
