@@ -455,13 +455,13 @@ kernel_fn pick_kernel(int ef_s, int* pool_slots) {
     return frog_search_kernel<16, MODE, BITMAP, F16>;
 }
 
-template <int ROWB>
+template <int ROWB, int MODE = MODE_FAST>
 kernel_fn pick_rowb(int ef_s) {
-    if (ef_s <= 32) return frog_search_kernel<1, MODE_FAST, true, false, ROWB>;
-    if (ef_s <= 64) return frog_search_kernel<2, MODE_FAST, true, false, ROWB>;
-    if (ef_s <= 128) return frog_search_kernel<4, MODE_FAST, true, false, ROWB>;
-    if (ef_s <= 256) return frog_search_kernel<8, MODE_FAST, true, false, ROWB>;
-    return frog_search_kernel<16, MODE_FAST, true, false, ROWB>;
+    if (ef_s <= 32) return frog_search_kernel<1, MODE, true, false, ROWB>;
+    if (ef_s <= 64) return frog_search_kernel<2, MODE, true, false, ROWB>;
+    if (ef_s <= 128) return frog_search_kernel<4, MODE, true, false, ROWB>;
+    if (ef_s <= 256) return frog_search_kernel<8, MODE, true, false, ROWB>;
+    return frog_search_kernel<16, MODE, true, false, ROWB>;
 }
 
 struct LaunchPlan {
@@ -491,6 +491,7 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
     if (P.eager_hash) {
         if (!bitmap || f16 || mode != MODE_FAST) return FROG_ERR_UNSUPPORTED;
         fn = pick_kernel<MODE_EAGER, true, false>(beam_width, &pool_slots);
+        if (ix->info.d_pad * 4 == 512) fn = pick_rowb<512, MODE_EAGER>(beam_width);
     }
     // common shapes with the row geometry fixed at compile time (fp32 rows of 384, 512 and 3072 bytes:
     // d = 96, 128, 768)
