@@ -219,6 +219,18 @@ __device__ __forceinline__ void tma_load_1d(void* dst_smem, const void* src_gmem
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
+// Four rows of a 2-D tensor (row-major rows of the vector store) in one request: the tensor map's
+// box is one row (or one column chunk of it) wide and one row high, the instruction names the first
+// column and four row indices, and the four pieces land back to back in shared memory (destination
+// 128-byte aligned).  Rows beyond the tensor read as zeros and still count their bytes.
+__device__ __forceinline__ void tma_gather4(void* dst_smem, const void* tensor_map, int col, int r0, int r1, int r2, int r3,
+                                            uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+                 ::"r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(tensor_map)), "r"(smem_u32(bar)),
+                   "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+                 : "memory");
+}
 // Wait for the phase of parity `phase`; bounded: gives up after 2^22 polls and reports false (the
 // caller flags the query instead of hanging the GPU).  try_wait already parks the thread for a
 // hardware-chosen interval per poll; passing an explicit suspend-time hint measured 7 % slower.
@@ -327,7 +339,9 @@ __device__ __forceinline__ float staged_dist2(const float* __restrict__ vectors,
 template <bool F16, int ROWB = 0>
 __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows, int row_bytes, int slot_bytes,
                                                    const float4* qs, float4* stage, uint64_t* bar,
-                                                   uint32_t& phases, bool& ok, uint32_t my_rank, int ns, int lane) {
+                                                   uint32_t& phases, bool& ok, uint32_t my_rank, int ns, int lane,
+                                                   const void* tmap = nullptr, const uint32_t* ranks = nullptr,
+                                                   int n_rows_total = 0) {
     if (ROWB > 0) {
         row_bytes = ROWB;
         slot_bytes = ROWB >= STAGE_CHUNK ? STAGE_CHUNK : ROWB;
@@ -340,17 +354,40 @@ __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows
     const int steps = ((ns + rph - 1) / rph) * chunks;
     const int team = lane >> 3, sub = lane & 7;
     int ig = 0, ic = 0;                                   // group and chunk of the next step to issue
+    // With a tensor map (`tmap`, `ranks` = the ns ranks in shared memory, 16-byte aligned) lane 0
+    // requests the rows of a step four at a time; slots past the last row name rows beyond the
+    // tensor (distinct ones), which arrive as zeros.  Otherwise one bulk copy per row.
+    constexpr int ELEM = F16 ? 2 : 4;
+    const int box_bytes = slot_bytes;                     // the box is one slot wide
     auto issue = [&](int s) {
         const int r0 = ig * rph, nrows = min(rph, ns - r0);
         const int c0 = ic * STAGE_CHUNK, cbytes = min(STAGE_CHUNK, row_bytes - c0);
         uint64_t* b = bar + (s & 1);
-        if (lane == 0) mbar_expect_tx(b, (uint32_t)(nrows * cbytes));
-        __syncwarp();
-        const uint32_t copy_rank = __shfl_sync(FULL, my_rank, (r0 + lane) & 31);
-        if (lane < nrows)
-            tma_load_1d(reinterpret_cast<char*>(stage) + (s & 1) * HALF + lane * slot_bytes,
-                        reinterpret_cast<const char*>(rows) + (size_t)copy_rank * (size_t)row_bytes + c0,
-                        (uint32_t)cbytes, b);
+        if (tmap) {
+            if (lane == 0) {
+                const int quads = (nrows + 3) >> 2;
+                mbar_expect_tx(b, (uint32_t)(quads * 4 * box_bytes));
+                char* dst = reinterpret_cast<char*>(stage) + (s & 1) * HALF;
+#pragma unroll
+                for (int qd = 0; qd < 2; ++qd) {
+                    if (qd < quads) {
+                        const uint4 rk = *reinterpret_cast<const uint4*>(ranks + r0 + 4 * qd);
+                        const int left = nrows - 4 * qd;        // valid rows of this quad (1..4)
+                        tma_gather4(dst + 4 * qd * slot_bytes, tmap, c0 / ELEM, (int)rk.x,
+                                    left > 1 ? (int)rk.y : n_rows_total + 1, left > 2 ? (int)rk.z : n_rows_total + 2,
+                                    left > 3 ? (int)rk.w : n_rows_total + 3, b);
+                    }
+                }
+            }
+        } else {
+            if (lane == 0) mbar_expect_tx(b, (uint32_t)(nrows * cbytes));
+            __syncwarp();
+            const uint32_t copy_rank = __shfl_sync(FULL, my_rank, (r0 + lane) & 31);
+            if (lane < nrows)
+                tma_load_1d(reinterpret_cast<char*>(stage) + (s & 1) * HALF + lane * slot_bytes,
+                            reinterpret_cast<const char*>(rows) + (size_t)copy_rank * (size_t)row_bytes + c0,
+                            (uint32_t)cbytes, b);
+        }
         if (++ic == chunks) { ic = 0; ++ig; }
     };
     issue(0);

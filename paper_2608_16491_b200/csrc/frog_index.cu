@@ -56,6 +56,7 @@ int alloc_device(frog_index* ix) {
     cudaDeviceProp prop;
     FROG_CUDA_TRY(cudaGetDeviceProperties(&prop, I.device));
     ix->sm_count = prop.multiProcessorCount;
+    ix->has_tmap_f32 = froghost::make_row_tensor_map(ix->d_vectors, false, I.d_pad, (size_t)I.d_pad * 4, n, &ix->tmap_f32);
     return FROG_OK;
 }
 

@@ -3,6 +3,7 @@
 
 #include <cstdint>
 #include <mutex>
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "frog.h"
@@ -35,6 +36,11 @@ struct frog_index {
     int n_scratch = 0;
     unsigned long long tick = 0;     // launch counter, for least-recently-used selection
     std::mutex mu;                   // guards the scratch sets and the order of launches into them
+    // Tensor maps of the two row stores for the 4-row gather of the copy engine (box = one row or
+    // one 512-byte column chunk of it); absent when the driver entry point is missing or the row
+    // shape does not qualify, in which case rows are copied one by one.
+    CUtensorMap tmap_f32, tmap_f16;
+    bool has_tmap_f32 = false, has_tmap_f16 = false;
     // staging for frog_search_host, grown on demand
     void* d_stage = nullptr;
     size_t stage_bytes = 0;
@@ -70,11 +76,14 @@ struct FrogSearchArgs {
     int row_bytes;             // bytes per stored row
     int slot_bytes;            // bytes of one row slot in the stage buffer (multiple of 16, <= 512)
     int q_len;                 // floats of the query held in shared memory (8 * ceil(d / 8))
+    int gather4;               // nonzero: `tmap` is valid and rows are fetched four per copy instruction
+    alignas(64) CUtensorMap tmap;
 };
 
 namespace froghost {
 void set_cuda_error(cudaError_t e);
 int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in, frog_params_t* out);
+bool make_row_tensor_map(const void* base, bool f16, int row_elems, size_t row_bytes, size_t n, CUtensorMap* out);
 int acquire_scratch(frog_index* ix, cudaStream_t s, FrogScratch** out);
 int ensure_bitmap(const frog_index* ix, FrogScratch* sc, size_t slots);
 int ensure_plan(FrogScratch* sc, size_t nq);

@@ -38,11 +38,16 @@ constexpr int WARPS_PER_CTA = FROG_WARPS_PER_CTA;
 #ifndef FROG_MINB_16
 #define FROG_MINB_16 10       // and of 512 entries (96 registers)
 #endif
+#ifndef FROG_GATHER4
+#define FROG_GATHER4 1         // rows fetched four per tensor-copy instruction where a tensor map exists
+#endif
 constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2, MODE_EAGER = 3;   // EAGER: FAST with the eager hash check
 
 constexpr int STAGE_BYTES = FROG_STAGE_ROWS * STAGE_CHUNK;
 
-// per-warp shared memory: pool | candidate list | two mbarriers, their parities, a failure flag | query | stage | hash
+// per-warp shared memory: stage | pool | candidate list | two mbarriers, their parities, a failure flag |
+// query | hash, the whole rounded up to 128 bytes (the stage buffer is the target of tensor copies,
+// which want 128-byte alignment)
 struct WarpSmem {
     uint64_t* pool;
     uint32_t* cand;
@@ -53,9 +58,10 @@ struct WarpSmem {
     uint32_t* hash;
 };
 
-inline size_t warp_smem_bytes(int pool_slots, int q_len, int hash_bits, bool bitmap) {
-    return (size_t)pool_slots * 8 + 64 * 4 + 32 + (size_t)q_len * 4 + STAGE_BYTES +
-           (bitmap ? 0 : ((size_t)4 << hash_bits));
+__host__ __device__ inline size_t warp_smem_bytes(int pool_slots, int q_len, int hash_bits, bool bitmap) {
+    const size_t b = (size_t)STAGE_BYTES + (size_t)pool_slots * 8 + 64 * 4 + 32 + (size_t)q_len * 4 +
+                     (bitmap ? 0 : ((size_t)4 << hash_bits));
+    return (b + 127) & ~(size_t)127;
 }
 inline int query_len(int d) { return (d + 7) / 8 * 8; }
 
@@ -92,7 +98,7 @@ template <int EPL, bool F16, int ROWB, bool UNIQUE>
 __device__ __noinline__ int evaluate_and_merge(const void* __restrict__ rows, int row_bytes, int slot_bytes, int ef_s,
                                                uint64_t* pool, const uint32_t* cand, uint64_t* bar,
                                                const float4* qs, float4* stage, int ns, uint32_t new_flag,
-                                               long long* t_dist) {
+                                               const void* tmap, int n, long long* t_dist) {
     const int lane = lane_id();
     uint32_t id = (lane < ns) ? cand[lane] : 0u;
     if (!UNIQUE) {
@@ -115,7 +121,8 @@ __device__ __noinline__ int evaluate_and_merge(const void* __restrict__ rows, in
         __syncwarp();                       // lane 0's update of the parity in the previous call
         uint32_t phase = bar_words[0];
         bool ok = true;
-        d2 = staged_dist2_pipe<F16, ROWB>(rows, row_bytes, slot_bytes, qs, stage, bar, phase, ok, id, ns, lane);
+        d2 = staged_dist2_pipe<F16, ROWB>(rows, row_bytes, slot_bytes, qs, stage, bar, phase, ok, id, ns, lane,
+                                          UNIQUE ? tmap : nullptr, cand, n);
         __syncwarp();                       // every lane has read the old parity
         if (lane == 0) {
             bar_words[0] = phase;
@@ -130,21 +137,20 @@ __device__ __noinline__ int evaluate_and_merge(const void* __restrict__ rows, in
 template <int EPL, int MODE, bool BITMAP, bool F16, int ROWB = 0>
 __global__ void __launch_bounds__(WARPS_PER_CTA * 32,
                                   (MODE == MODE_FAST || MODE == MODE_EAGER) ? (EPL <= 4 ? FROG_MINB : EPL == 8 ? FROG_MINB_8 : FROG_MINB_16) : 1)
-frog_search_kernel(const FrogSearchArgs A) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     const int lane = lane_id();
     const int warp = threadIdx.x >> 5;
     constexpr int POOL = 32 * EPL;
     const int hash_slots = BITMAP ? 0 : (1 << A.hash_bits);
-    const size_t per_warp = (size_t)POOL * 8 + 64 * 4 + 32 + (size_t)A.q_len * 4 + STAGE_BYTES + (size_t)hash_slots * 4;
-    unsigned char* base = smem_raw + per_warp * warp;
+    unsigned char* base = smem_raw + warp_smem_bytes(POOL, A.q_len, A.hash_bits, BITMAP) * warp;
     WarpSmem S;
-    S.pool = reinterpret_cast<uint64_t*>(base);
+    S.stage = reinterpret_cast<float4*>(base);
+    S.pool = reinterpret_cast<uint64_t*>(base + STAGE_BYTES);
     S.cand = reinterpret_cast<uint32_t*>(S.pool + POOL);
     S.bar = reinterpret_cast<uint64_t*>(S.cand + 64);
     S.q = reinterpret_cast<float4*>(S.bar + 4);
-    S.stage = reinterpret_cast<float4*>(reinterpret_cast<float*>(S.q) + A.q_len);
-    S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(S.stage) + STAGE_BYTES);
+    S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<float*>(S.q) + A.q_len);
     if (lane == 0) {
         mbar_init(S.bar, 1u);
         mbar_init(S.bar + 1, 1u);
@@ -180,6 +186,7 @@ frog_search_kernel(const FrogSearchArgs A) {
         auto EVAL = [&](int ns_, uint32_t flag_, int off_ = 0) {
             int f_ = evaluate_and_merge<EPL, F16, ROWB, BITMAP>(A.rows, A.row_bytes, A.slot_bytes, A.ef_s, S.pool,
                                                   S.cand + off_, S.bar, S.q, S.stage, ns_, flag_,
+                                                  A.gather4 ? &A.tmap : nullptr, A.n,
                                                   MODE == MODE_PROFILE ? &t_split : nullptr);
             if (MODE == MODE_PROFILE) {
                 long long n_ = clock64();
@@ -527,6 +534,9 @@ void set_gather(const frog_index* ix, bool f16, FrogSearchArgs* A) {
     A->row_bytes = f16 ? d_pad_h * 2 : ix->info.d_pad * 4;
     A->slot_bytes = A->row_bytes < STAGE_CHUNK ? A->row_bytes : STAGE_CHUNK;   // rows are 16-byte multiples
     A->q_len = d_pad_h;
+    A->gather4 = FROG_GATHER4 && (f16 ? ix->has_tmap_f16 : ix->has_tmap_f32);
+    if (A->gather4) A->tmap = f16 ? ix->tmap_f16 : ix->tmap_f32;
+    else std::memset(&A->tmap, 0, sizeof(A->tmap));
 }
 
 // per-warp visited slab: one bit per rank, padded to 128 bytes
@@ -564,6 +574,42 @@ int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in
     (void)ix;
     *out = P;
     return FROG_OK;
+}
+
+// Tensor map over a row store (n rows of row_elems elements, row_bytes apart) whose box is one row
+// high and one stage slot wide: what the 4-row gather of the copy engine needs.  Returns false
+// (rows are then copied one by one) if the driver entry point cannot be had, the shape does not
+// qualify (two quads per stage half need 4 slots to be a multiple of 128 bytes) or encoding fails.
+bool make_row_tensor_map(const void* base, bool f16, int row_elems, size_t row_bytes, size_t n, CUtensorMap* out) {
+    typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn encode = nullptr;
+    static bool looked_up = false;
+    if (!looked_up) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            encode = reinterpret_cast<encode_fn>(fn);
+        else
+            cudaGetLastError();
+        looked_up = true;
+    }
+    const int elem = f16 ? 2 : 4;
+    const size_t slot = row_bytes < (size_t)STAGE_CHUNK ? row_bytes : (size_t)STAGE_CHUNK;
+    if (!encode || !base || n == 0 || n > 0x7FFFFFF0ull) return false;
+    if (row_bytes % 16 != 0 || slot % 16 != 0 || (reinterpret_cast<uintptr_t>(base) & 15) != 0) return false;
+    if (slot <= 256 && slot % 32 != 0) return false;
+    cuuint64_t gdim[2] = {(cuuint64_t)row_elems, (cuuint64_t)n};
+    cuuint64_t gstride[1] = {(cuuint64_t)row_bytes};
+    cuuint32_t box[2] = {(cuuint32_t)(slot / elem), 1u};
+    cuuint32_t estride[2] = {1u, 1u};
+    const CUresult r = encode(out, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                              const_cast<void*>(base), gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
 }
 
 // Scratch set for a launch on stream s.  Launches of one stream are ordered by the stream, so a
@@ -900,5 +946,7 @@ extern "C" int frog_index_enable_f16(frog_index_t* ix) {
     FROG_CUDA_TRY(cudaGetLastError());
     FROG_CUDA_TRY(cudaDeviceSynchronize());
     ix->info.device_bytes += (int64_t)(elems * sizeof(__half));
+    ix->has_tmap_f16 = froghost::make_row_tensor_map(ix->d_vectors_h, true, d_pad_h, (size_t)d_pad_h * 2,
+                                                     (size_t)ix->info.n, &ix->tmap_f16);
     return FROG_OK;
 }
