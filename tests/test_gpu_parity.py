@@ -307,6 +307,32 @@ def test_odd_dimension(libs, cache_dir):
     gix.close()
 
 
+@pytest.mark.parametrize("n,d,m,n_inv", [(1, 8, 16, 7), (2, 16, 16, 7), (33, 24, 16, 3), (200, 40, 8, 4),
+                                          (1000, 64, 32, 5), (777, 12, 4, 2)])
+def test_small_and_odd_indexes(libs, cache_dir, n, d, m, n_inv):
+    """Degenerate index shapes: a single object, fewer objects than a warp, one retained layer,
+    row sizes that do and do not qualify for the 4-row tensor gather (slots of 32, 64, 96, 160, 256
+    and 48 bytes), several ENC widths."""
+    rng = np.random.default_rng(100 + n)
+    V = rng.standard_normal((n, d)).astype(np.float32)
+    a = rng.integers(0, max(2, n // 2), n).astype(np.int32)
+    path = os.path.join(cache_dir, f"small_{n}_{d}_{m}.idx")
+    libs.build_index(V, a, path, m=m, n_inv=n_inv, ef_c=64)
+    ix = oracle.load_index(path)
+    gix = libs.Index.load(path, 0)
+    try:
+        nq = 96
+        Q = rng.standard_normal((nq, d)).astype(np.float32)
+        lo = rng.integers(-2, max(2, n // 2), nq).astype(np.int32)
+        hi = (lo + rng.integers(0, max(2, n // 2) + 2, nq)).astype(np.int32)
+        for k, ef, B in ((1, 8, 16), (5, 16, 64), (10, 48, 33)):
+            ref = oracle.search(ix, Q, lo, hi, k, ef, B=B)
+            got = _gpu_search(libs, gix, Q, lo, hi, k, ef, budget=B)
+            _assert_parity(got, ref)
+    finally:
+        gix.close()
+
+
 def test_index_info_and_from_host(libs, tiny):
     wl, path, ix = tiny
     gix = libs.Index.load(path, 0)
