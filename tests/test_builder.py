@@ -30,6 +30,29 @@ def test_fusion_distance_limits_and_monotonicity(libs):
         assert (f(xx, zx, 0.2, 0.5) < f(xy, zy, 0.2, 0.5)) == (xx / xy < w(zy) / w(zx))
 
 
+def test_fusion_distance_first_order_shift_of_attribute_distance(libs):
+    """Sec. 5.2: keeping the q-fraction of candidates with the smallest fusion distance lowers the
+    mean attribute distance of the kept ones by alpha * beta * C_gamma to first order in beta, with
+    C_gamma = gamma / (2 (gamma + 1)(gamma + 2)) for Z ~ U(0,1), when X and Z are independent and
+    F_X(x) ~ x^alpha near 0.  Monte Carlo with X = U^(1/alpha) (F_X(x) = x^alpha exactly)."""
+    f = libs.fusion_distance
+    rng = np.random.default_rng(11)
+    N, q, alpha, gamma = 400_000, 0.02, 2.0, 0.5
+    X = rng.uniform(0, 1, N) ** (1.0 / alpha)
+    Z = rng.uniform(0, 1, N)
+    c_gamma = gamma / (2 * (gamma + 1) * (gamma + 2))
+    keep = int(q * N)
+    base = Z[np.argsort(X)[:keep]].mean()                   # beta = 0: selection ignores Z
+    assert abs(base - 0.5) < 0.01
+    shifts = {}
+    for beta in (0.05, 0.1):
+        Y = np.fromiter((f(float(x), float(z), beta, gamma) for x, z in zip(X, Z)), dtype=np.float64, count=N)
+        shifts[beta] = base - Z[np.argsort(Y)[:keep]].mean()
+        predicted = alpha * beta * c_gamma
+        assert 0.7 * predicted < shifts[beta] < 1.4 * predicted, (beta, shifts[beta], predicted)
+    assert shifts[0.1] > 1.6 * shifts[0.05]                 # first order in beta
+
+
 def test_retained_depth(libs):
     # H = ceil(log2 n) + 1 - n_inv
     assert libs.retained_depth(10_000, 7) == 8
