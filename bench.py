@@ -392,7 +392,7 @@ def run_ours(args):
 
     # ---- CPU oracle on the host cores, bounded sample; doubles as a parity check ------------------
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and ws == 1:      # rank 0 at N = 1 only
         import oracle
         oix = oracle.load_index(path)
         S = min(args.cpu_sample, nq)
