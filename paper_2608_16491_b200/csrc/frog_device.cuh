@@ -36,6 +36,32 @@ __device__ __forceinline__ uint32_t ldg_stream_u32(const uint32_t* p) {
     asm("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
     return v;
 }
+// L2 eviction policies for a whole access.  Short vector rows are read about once per batch and
+// should leave L2 first (long rows are kept at normal priority: their popular rows are worth
+// 4 % when they stay); the visited slab of a query is hit again and again and should stay.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_normal() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint32_t atomic_or_l2(uint32_t* p, uint32_t v, uint64_t policy) {
+    uint32_t old;
+    asm volatile("atom.global.or.b32.L2::cache_hint %0, [%1], %2, %3;" : "=r"(old) : "l"(p), "r"(v), "l"(policy) : "memory");
+    return old;
+}
+__device__ __forceinline__ void st_u32_l2(uint32_t* p, uint32_t v, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.u32 [%0], %1, %2;" ::"l"(p), "r"(v), "l"(policy) : "memory");
+}
 
 // Pool key: (squared distance bits) << 32 | rank << 1 | expanded flag.  Distances are >= +0, so
 // the fp32 bit pattern is monotone as an unsigned integer; ranks are unique, so comparing
@@ -224,12 +250,18 @@ __device__ __forceinline__ void tma_load_1d(void* dst_smem, const void* src_gmem
 // column and four row indices, and the four pieces land back to back in shared memory (destination
 // 128-byte aligned).  Rows beyond the tensor read as zeros and still count their bytes.
 __device__ __forceinline__ void tma_gather4(void* dst_smem, const void* tensor_map, int col, int r0, int r1, int r2, int r3,
-                                            uint64_t* bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
-                 " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+                                            uint64_t* bar, uint64_t l2_policy) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes.L2::cache_hint"
+                 " [%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;"
                  ::"r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(tensor_map)), "r"(smem_u32(bar)),
-                   "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+                   "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "l"(l2_policy)
                  : "memory");
+}
+// tma_load_1d with an L2 eviction policy
+__device__ __forceinline__ void tma_load_1d_l2(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar,
+                                               uint64_t l2_policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)), "l"(l2_policy) : "memory");
 }
 // Wait for the phase of parity `phase`; bounded: gives up after 2^22 polls and reports false (the
 // caller flags the query instead of hanging the GPU).  try_wait already parks the thread for a
@@ -359,6 +391,7 @@ __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows
     // tensor (distinct ones), which arrive as zeros.  Otherwise one bulk copy per row.
     constexpr int ELEM = F16 ? 2 : 4;
     const int box_bytes = slot_bytes;                     // the box is one slot wide
+    const uint64_t row_policy = row_bytes <= STAGE_CHUNK ? l2_policy_evict_first() : l2_policy_evict_normal();
     auto issue = [&](int s) {
         const int r0 = ig * rph, nrows = min(rph, ns - r0);
         const int c0 = ic * STAGE_CHUNK, cbytes = min(STAGE_CHUNK, row_bytes - c0);
@@ -375,7 +408,7 @@ __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows
                         const int left = nrows - 4 * qd;        // valid rows of this quad (1..4)
                         tma_gather4(dst + 4 * qd * slot_bytes, tmap, c0 / ELEM, (int)rk.x,
                                     left > 1 ? (int)rk.y : n_rows_total + 1, left > 2 ? (int)rk.z : n_rows_total + 2,
-                                    left > 3 ? (int)rk.w : n_rows_total + 3, b);
+                                    left > 3 ? (int)rk.w : n_rows_total + 3, b, row_policy);
                     }
                 }
             }
@@ -384,9 +417,9 @@ __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows
             __syncwarp();
             const uint32_t copy_rank = __shfl_sync(FULL, my_rank, (r0 + lane) & 31);
             if (lane < nrows)
-                tma_load_1d(reinterpret_cast<char*>(stage) + (s & 1) * HALF + lane * slot_bytes,
-                            reinterpret_cast<const char*>(rows) + (size_t)copy_rank * (size_t)row_bytes + c0,
-                            (uint32_t)cbytes, b);
+                tma_load_1d_l2(reinterpret_cast<char*>(stage) + (s & 1) * HALF + lane * slot_bytes,
+                               reinterpret_cast<const char*>(rows) + (size_t)copy_rank * (size_t)row_bytes + c0,
+                               (uint32_t)cbytes, b, row_policy);
         }
         if (++ic == chunks) { ic = 0; ++ig; }
     };

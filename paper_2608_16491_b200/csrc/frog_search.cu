@@ -160,6 +160,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
     __syncwarp();
     uint32_t* bitmap = BITMAP ? A.bitmap + (size_t)(blockIdx.x * WARPS_PER_CTA + warp) * A.bitmap_words : nullptr;
     const uint32_t lt_mask = (1u << lane) - 1u;
+    const uint64_t keep_in_l2 = l2_policy_evict_last();      // for the visited slab of the running query
 
     for (;;) {
         int q = 0;
@@ -237,7 +238,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
             if (BITMAP) {
                 // clear the words that cover [l_q, r_q]
                 const int w0 = l_q >> 5, w1 = r_q >> 5;
-                for (int i = w0 + lane; i <= w1; i += 32) bitmap[i] = 0u;
+                for (int i = w0 + lane; i <= w1; i += 32) st_u32_l2(bitmap + i, 0u, keep_in_l2);
             } else {
                 uint4* h4 = reinterpret_cast<uint4*>(S.hash);
                 const uint4 e4 = make_uint4(HASH_EMPTY, HASH_EMPTY, HASH_EMPTY, HASH_EMPTY);
@@ -334,8 +335,8 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                     if (BITMAP) {
                         const uint32_t bit0 = 1u << (v0 & 31), bit1 = 1u << (v1 & 31);
                         uint32_t old0 = 0xFFFFFFFFu, old1 = 0xFFFFFFFFu;
-                        if (adm0) old0 = atomicOr(bitmap + (v0 >> 5), bit0);
-                        if (adm1) old1 = atomicOr(bitmap + (v1 >> 5), bit1);
+                        if (adm0) old0 = atomic_or_l2(bitmap + (v0 >> 5), bit0, keep_in_l2);
+                        if (adm1) old1 = atomic_or_l2(bitmap + (v1 >> 5), bit1, keep_in_l2);
                         keep0 = (old0 & bit0) == 0;
                         keep1 = (old1 & bit1) == 0;
                     } else {
