@@ -307,49 +307,80 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                         scanned = min(total, c0 + 32);
                     }
                 } else
-                for (int c0 = 0; c0 < total && cnt < A.B; c0 += 64) {
-                    uint32_t v0 = BOT, v1 = BOT;
+                // Four 32-entry chunks are fetched per round trip and their visited atomics are in
+                // flight together; the admission under budget B runs over them in order, so the EN
+                // list is the one a chunk-by-chunk scan yields.  A chunk counts as scanned only if it
+                // exists and budget is left after the chunks before it.
+                for (int c0 = 0; c0 < total && cnt < A.B; c0 += 128) {
+                    uint32_t v0 = BOT, v1 = BOT, v2 = BOT, v3 = BOT;
                     if (c0 + lane < total) v0 = ldg_stream_u32(hot + c0 + lane);
                     if (c0 + 32 + lane < total) v1 = ldg_stream_u32(hot + c0 + 32 + lane);
-                    // first chunk
+                    if (c0 + 64 + lane < total) v2 = ldg_stream_u32(hot + c0 + 64 + lane);
+                    if (c0 + 96 + lane < total) v3 = ldg_stream_u32(hot + c0 + 96 + lane);
                     const bool pred0 = (v0 - (uint32_t)l_q) <= span;
                     const uint32_t M0 = __ballot_sync(FULL, pred0);
                     const int a0 = min(__popc(M0), A.B - cnt);
                     const int rank0 = __popc(M0 & lt_mask);
                     const bool adm0 = pred0 && rank0 < a0;
-                    // second chunk: scanned only if budget is left after the first
-                    const int rem = A.B - cnt - a0;
-                    const bool has1 = (c0 + 32 < total) && rem > 0;
+                    const int rem1 = A.B - cnt - a0;
+                    const bool has1 = (c0 + 32 < total) && rem1 > 0;
                     const bool pred1 = has1 && ((v1 - (uint32_t)l_q) <= span);
                     const uint32_t M1 = __ballot_sync(FULL, pred1);
-                    const int a1 = min(__popc(M1), rem);
+                    const int a1 = min(__popc(M1), rem1);
                     const int rank1 = __popc(M1 & lt_mask);
                     const bool adm1 = pred1 && rank1 < a1;
+                    const int rem2 = rem1 - a1;
+                    const bool has2 = (c0 + 64 < total) && rem2 > 0;
+                    const bool pred2 = has2 && ((v2 - (uint32_t)l_q) <= span);
+                    const uint32_t M2 = __ballot_sync(FULL, pred2);
+                    const int a2 = min(__popc(M2), rem2);
+                    const int rank2 = __popc(M2 & lt_mask);
+                    const bool adm2 = pred2 && rank2 < a2;
+                    const int rem3 = rem2 - a2;
+                    const bool has3 = (c0 + 96 < total) && rem3 > 0;
+                    const bool pred3 = has3 && ((v3 - (uint32_t)l_q) <= span);
+                    const uint32_t M3 = __ballot_sync(FULL, pred3);
+                    const int a3 = min(__popc(M3), rem3);
+                    const int rank3 = __popc(M3 & lt_mask);
+                    const bool adm3 = pred3 && rank3 < a3;
                     if (MODE == MODE_TRACE && rec_ok) {
                         if (adm0) trace_row[3 + trace_len + cnt + rank0] = v0;
                         if (adm1) trace_row[3 + trace_len + cnt + a0 + rank1] = v1;
+                        if (adm2) trace_row[3 + trace_len + cnt + a0 + a1 + rank2] = v2;
+                        if (adm3) trace_row[3 + trace_len + cnt + a0 + a1 + a2 + rank3] = v3;
                     }
                     FROG_PHASE(1);
-                    // visited check of both chunks; with the bitmap the two atomics are in flight together
-                    bool keep0, keep1;
+                    bool keep0, keep1, keep2, keep3;
                     if (BITMAP) {
                         const uint32_t bit0 = 1u << (v0 & 31), bit1 = 1u << (v1 & 31);
-                        uint32_t old0 = 0xFFFFFFFFu, old1 = 0xFFFFFFFFu;
+                        const uint32_t bit2 = 1u << (v2 & 31), bit3 = 1u << (v3 & 31);
+                        uint32_t old0 = 0xFFFFFFFFu, old1 = 0xFFFFFFFFu, old2 = 0xFFFFFFFFu, old3 = 0xFFFFFFFFu;
                         if (adm0) old0 = atomic_or_l2(bitmap + (v0 >> 5), bit0, keep_in_l2);
                         if (adm1) old1 = atomic_or_l2(bitmap + (v1 >> 5), bit1, keep_in_l2);
+                        if (adm2) old2 = atomic_or_l2(bitmap + (v2 >> 5), bit2, keep_in_l2);
+                        if (adm3) old3 = atomic_or_l2(bitmap + (v3 >> 5), bit3, keep_in_l2);
                         keep0 = (old0 & bit0) == 0;
                         keep1 = (old1 & bit1) == 0;
+                        keep2 = (old2 & bit2) == 0;
+                        keep3 = (old3 & bit3) == 0;
                     } else {
                         keep0 = adm0 && visited_insert(S.hash, A.hash_bits, v0, forgets);
                         keep1 = adm1 && visited_insert(S.hash, A.hash_bits, v1, forgets);
+                        keep2 = adm2 && visited_insert(S.hash, A.hash_bits, v2, forgets);
+                        keep3 = adm3 && visited_insert(S.hash, A.hash_bits, v3, forgets);
                     }
                     const uint32_t K0 = __ballot_sync(FULL, keep0);
                     const uint32_t K1 = __ballot_sync(FULL, keep1);
+                    const uint32_t K2 = __ballot_sync(FULL, keep2);
+                    const uint32_t K3 = __ballot_sync(FULL, keep3);
+                    const int n0 = __popc(K0), n1 = __popc(K1), n2 = __popc(K2);
                     if (keep0) S.cand[ns + __popc(K0 & lt_mask)] = v0;
-                    if (keep1) S.cand[ns + __popc(K0) + __popc(K1 & lt_mask)] = v1;
-                    ns += __popc(K0) + __popc(K1);
-                    cnt += a0 + a1;
-                    scanned = min(total, c0 + (has1 ? 64 : 32));
+                    if (keep1) S.cand[ns + n0 + __popc(K1 & lt_mask)] = v1;
+                    if (keep2) S.cand[ns + n0 + n1 + __popc(K2 & lt_mask)] = v2;
+                    if (keep3) S.cand[ns + n0 + n1 + n2 + __popc(K3 & lt_mask)] = v3;
+                    ns += n0 + n1 + n2 + __popc(K3);
+                    cnt += a0 + a1 + a2 + a3;
+                    scanned = min(total, c0 + (has3 ? 128 : has2 ? 96 : has1 ? 64 : 32));
                     FROG_PHASE(2);
                 }
                 __syncwarp();
