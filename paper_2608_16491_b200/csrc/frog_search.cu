@@ -41,7 +41,8 @@ constexpr int WARPS_PER_CTA = FROG_WARPS_PER_CTA;
 #ifndef FROG_GATHER4
 #define FROG_GATHER4 1         // rows fetched four per tensor-copy instruction where a tensor map exists
 #endif
-constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2, MODE_EAGER = 3;   // EAGER: FAST with the eager hash check
+constexpr int MODE_FAST = 0, MODE_TRACE = 1, MODE_PROFILE = 2, MODE_EAGER = 3, MODE_COUNT = 4;
+// EAGER: FAST with the eager hash check; COUNT: FAST that also keeps the per-query counters (`stats`)
 
 constexpr int STAGE_BYTES = FROG_STAGE_ROWS * STAGE_CHUNK;
 
@@ -136,7 +137,8 @@ __device__ __noinline__ int evaluate_and_merge(const void* __restrict__ rows, in
 
 template <int EPL, int MODE, bool BITMAP, bool F16, int ROWB = 0>
 __global__ void __launch_bounds__(WARPS_PER_CTA * 32,
-                                  (MODE == MODE_FAST || MODE == MODE_EAGER) ? (EPL <= 4 ? FROG_MINB : EPL == 8 ? FROG_MINB_8 : FROG_MINB_16) : 1)
+                                  (MODE == MODE_FAST || MODE == MODE_EAGER || MODE == MODE_COUNT)
+                                      ? (EPL <= 4 ? FROG_MINB : EPL == 8 ? FROG_MINB_8 : FROG_MINB_16) : 1)
 frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int lane = lane_id();
@@ -215,6 +217,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
             warp_rank_interval(A.sorted_attr, A.n, lo, hi, lane, l_q, r_q);    // Sec. 4
         }
         const int w = (lo > hi) ? 0 : (r_q - l_q + 1);
+        constexpr bool COUNT = MODE != MODE_FAST;          // the plain kernel keeps no work counters
         uint32_t st = 0, n_exp = 0, n_rows = 0, n_en = 0, n_dist = 0, forgets = 0;
         uint32_t trace_len = 0;
         bool trace_ok = true;
@@ -231,7 +234,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                 if (lane < cnt) S.cand[lane] = (uint32_t)(l_q + b0 + lane);
                 __syncwarp();
                 EVAL(cnt, 1u);
-                n_dist += cnt;
+                if (COUNT) n_dist += cnt;
                 __syncwarp();
             }
         } else {
@@ -262,7 +265,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                 __syncwarp();
             }
             FROG_PHASE(0);
-            n_dist += ns;
+            if (COUNT) n_dist += ns;
             int first = EVAL(ns, 0u);
             // lines 7-17
             while (first < A.ef_s) {
@@ -380,14 +383,16 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                     if (keep3) S.cand[ns + n0 + n1 + n2 + __popc(K3 & lt_mask)] = v3;
                     ns += n0 + n1 + n2 + __popc(K3);
                     cnt += a0 + a1 + a2 + a3;
-                    scanned = min(total, c0 + (has3 ? 128 : has2 ? 96 : has1 ? 64 : 32));
+                    if (COUNT) scanned = min(total, c0 + (has3 ? 128 : has2 ? 96 : has1 ? 64 : 32));
                     FROG_PHASE(2);
                 }
                 __syncwarp();
                 ++n_exp;
-                n_rows += (scanned + A.m - 1) / A.m;
-                n_en += cnt;
-                n_dist += ns;
+                if (COUNT) {
+                    n_rows += (scanned + A.m - 1) / A.m;
+                    n_en += cnt;
+                    n_dist += ns;
+                }
                 if (MODE == MODE_TRACE) {
                     if (rec_ok) {
                         if (lane == 0) { trace_row[1 + trace_len] = u; trace_row[2 + trace_len] = (uint32_t)cnt; }
@@ -429,7 +434,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
         FROG_PHASE(4);
         if (lane == 0) {
             if (A.status) A.status[q] = st;
-            if (A.stats) {
+            if (COUNT && A.stats) {
                 uint32_t* srow = A.stats + 4 * (size_t)q;
                 srow[0] = n_exp; srow[1] = n_rows; srow[2] = n_en; srow[3] = n_dist;
             }
@@ -518,17 +523,20 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
     if (f16)
         fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, true, true>(beam_width, &pool_slots)
            : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, true, true>(beam_width, &pool_slots)
-                                  : pick_kernel<MODE_FAST, true, true>(beam_width, &pool_slots);
+           : mode == MODE_COUNT ? pick_kernel<MODE_COUNT, true, true>(beam_width, &pool_slots)
+                                : pick_kernel<MODE_FAST, true, true>(beam_width, &pool_slots);
     else if (bitmap)
         fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, true, false>(beam_width, &pool_slots)
            : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, true, false>(beam_width, &pool_slots)
-                                  : pick_kernel<MODE_FAST, true, false>(beam_width, &pool_slots);
+           : mode == MODE_COUNT ? pick_kernel<MODE_COUNT, true, false>(beam_width, &pool_slots)
+                                : pick_kernel<MODE_FAST, true, false>(beam_width, &pool_slots);
     else
         fn = mode == MODE_TRACE ? pick_kernel<MODE_TRACE, false, false>(beam_width, &pool_slots)
            : mode == MODE_PROFILE ? pick_kernel<MODE_PROFILE, false, false>(beam_width, &pool_slots)
-                                  : pick_kernel<MODE_FAST, false, false>(beam_width, &pool_slots);
+           : mode == MODE_COUNT ? pick_kernel<MODE_COUNT, false, false>(beam_width, &pool_slots)
+                                : pick_kernel<MODE_FAST, false, false>(beam_width, &pool_slots);
     if (P.eager_hash) {
-        if (!bitmap || f16 || mode != MODE_FAST) return FROG_ERR_UNSUPPORTED;
+        if (!bitmap || f16 || (mode != MODE_FAST && mode != MODE_COUNT)) return FROG_ERR_UNSUPPORTED;
         fn = pick_kernel<MODE_EAGER, true, false>(beam_width, &pool_slots);
         if (ix->info.d_pad * 4 == 512) fn = pick_rowb<512, MODE_EAGER>(beam_width);
     }
@@ -752,7 +760,7 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     int rc = froghost::resolve_params(index, beam_width, params, &P);
     if (rc) return rc;
     FROG_CUDA_TRY(cudaSetDevice(index->info.device));
-    const int mode = !trace ? MODE_FAST : (P.debug_flags & 1) ? MODE_PROFILE : MODE_TRACE;
+    const int mode = trace ? ((P.debug_flags & 1) ? MODE_PROFILE : MODE_TRACE) : stats ? MODE_COUNT : MODE_FAST;
     bool bitmap = P.visited != FROG_VISITED_HASH;
     LaunchPlan plan;
     rc = plan_launch(index, beam_width, P, mode, bitmap, nq, &plan);

@@ -25,6 +25,10 @@ def _gpu_search(frog, gix, wl_q, lo, hi, k, ef, trace_cap=0, **params):
     p = frog.Params(**params) if params else None
     ids, dists = gix.search(q, tlo, thi, k, ef, params=p, status=status, stats=stats, trace=trace)
     torch.cuda.synchronize()
+    # the plain kernel (no counters, no trace) must give the same answers
+    ids2, dists2 = gix.search(q, tlo, thi, k, ef, params=p)
+    torch.cuda.synchronize()
+    assert torch.equal(ids, ids2) and torch.equal(dists.view(torch.int32), dists2.view(torch.int32))   # bit for bit
     return (ids.cpu().numpy(), dists.cpu().numpy(), status.cpu().numpy().view(np.uint32),
             stats.cpu().numpy().view(np.uint32), None if trace is None else trace.cpu().numpy().view(np.uint32))
 
