@@ -37,7 +37,7 @@ RECALL_TARGET = 0.95
 HBM_FALLBACK_GBS = 6650.0
 # DRAM bytes of one search-kernel launch at the default bench point (sift 1M, B = 64, ef_s = 44),
 # from the ncu capture summarised in profiles/frog_search_kernel_sift1m_b64_ef44.md
-NCU_TRAFFIC = {("sift", 1_000_000, 64, 44): 5.175e9}
+NCU_TRAFFIC = {("sift", 1_000_000, 64, 44): 5.434e9}
 
 
 def log(*a):
