@@ -154,7 +154,8 @@ int frog_search(const frog_index_t* index, const float* queries, const int32_t* 
  *   params  HOST, may be null (defaults)
  *   status  DEVICE nq uint32 or null: FROG_ST_* bits
  *   stats   DEVICE nq x 4 uint32 or null: {expansions, ENC rows the scan needed, ENs admitted
- *           by Alg. 4, distance evaluations}
+ *           by Alg. 4, distance evaluations}.  Asking for them selects a variant of the kernel
+ *           that keeps these counters (a few per cent slower than the plain one; same results)
  *   trace   DEVICE nq x trace_cap uint32 or null: row q = [len, then per expansion
  *           u, |EN(u)|, EN(u)[0..]] (ranks); records are appended while at least 66 words
  *           remain in the row.  Selects a slower kernel instantiation; meant for tests. */
