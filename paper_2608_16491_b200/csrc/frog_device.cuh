@@ -524,6 +524,33 @@ __device__ __forceinline__ uint32_t merge_batch(uint64_t* pool, uint64_t my_key,
     bool dropped = false;
     const uint32_t my_lo = (uint32_t)my_key | 1u, my_hi = (uint32_t)(my_key >> 32);
     const uint64_t mk = my_key | 1ull;
+    if (UNIQUE && EPL <= 4) {
+        // no copies to look for: two entering keys per iteration, so that the shuffles and ballots
+        // of one overlap those of the other (the chain of one key at a time is latency, not work)
+#pragma unroll 1
+        for (uint32_t msk = have; msk;) {
+            const int j0 = __ffs(msk) - 1;
+            msk &= msk - 1;
+            const int j1 = msk ? __ffs(msk) - 1 : j0;
+            const bool two = msk != 0;
+            msk &= msk - 1;
+            const uint64_t x0 = ((uint64_t)__shfl_sync(FULL, my_hi, j0) << 32) | __shfl_sync(FULL, my_lo, j0);
+            uint64_t x1 = ((uint64_t)__shfl_sync(FULL, my_hi, j1) << 32) | __shfl_sync(FULL, my_lo, j1);
+            if (!two) x1 = KEY_EMPTY;                       // compares below nothing
+            int above0 = 0, above1 = 0;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) {
+                const uint64_t p = pk[e] | 1ull;
+                const bool lt0 = x0 < p, lt1 = x1 < p;
+                above0 += __popc(__ballot_sync(FULL, lt0));
+                above1 += __popc(__ballot_sync(FULL, lt1));
+                add[e] += (lt0 ? 1 : 0) + (lt1 ? 1 : 0);
+            }
+            rnew += ((x0 < mk) ? 1 : 0) + ((x1 < mk) ? 1 : 0);
+            if (lane == j0) above = above0;
+            if (two && lane == j1) above = above1;
+        }
+    } else
 #pragma unroll 1
     for (uint32_t msk = have; msk; msk &= msk - 1) {
         const int j = __ffs(msk) - 1;
