@@ -273,7 +273,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                 const uint32_t u = key_rank(S.pool[first]);               // line 8
                 __syncwarp();
                 if (lane == 0) S.pool[first] |= 1ull;                     // line 9
-                // line 10, Alg. 4: scan rows L_start..L_end of ENC(u) in 32-entry chunks (two
+                // line 10, Alg. 4: scan rows L_start..L_end of ENC(u) in 32-entry chunks (four
                 // fetched per round trip); predicate "not empty and l_q <= v <= r_q" as one
                 // unsigned compare (the empty entry 0xFFFFFFFF minus l_q exceeds any span);
                 // ballot + popc give the admitted prefix under budget B.  Lines 12-13: each
