@@ -62,8 +62,26 @@ def _load(path: str) -> C.CDLL:
     return C.CDLL(path)
 
 
-_lib = _load(_LIB_SEARCH)
-_lib.frog_strerror.restype = C.c_char_p
+class _SearchLib:
+    """libfrog.so, loaded at the first use of any of its functions.  Importing the package must work
+    on a fresh checkout (the build step lives in this package); every call into the search path
+    without the compiled library raises ImportError — there is nothing to fall back to."""
+
+    def __init__(self):
+        self._dll = None
+
+    def _get(self) -> C.CDLL:
+        if self._dll is None:
+            dll = _load(_LIB_SEARCH)
+            dll.frog_strerror.restype = C.c_char_p
+            self._dll = dll
+        return self._dll
+
+    def __getattr__(self, name):
+        return getattr(self._get(), name)
+
+
+_lib = _SearchLib()
 _blib = None
 
 _vp = C.c_void_p
