@@ -50,3 +50,26 @@ def test_loader_rejects_malformed_files(libs, tmp_path):
     assert frog._lib.frog_index_load(str(p).encode(), 0, ctypes.byref(h)) == 3
     p.write_bytes(b"FROG")
     assert frog._lib.frog_index_load(str(p).encode(), 0, ctypes.byref(h)) == 3
+
+
+def test_missing_library_fails_loudly_at_first_use(tmp_path):
+    """The package imports without the compiled search library (its build step lives in it), but
+    every call into the search path then raises: there is no fallback implementation."""
+    import subprocess
+    import sys
+    code = (
+        "import os, sys\n"
+        "sys.path.insert(0, %r)\n"
+        "os.environ['FROG_LIBFROG'] = %r\n"
+        "import paper_2608_16491_b200 as frog\n"
+        "from paper_2608_16491_b200 import build\n"
+        "try:\n"
+        "    frog.strerror(0)\n"
+        "except ImportError as e:\n"
+        "    print('LOUD', 'no fallback' in str(e))\n"
+        "else:\n"
+        "    print('SILENT')\n"
+    ) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), str(tmp_path / "nowhere" / "libfrog.so"))
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=120)
+    assert out.returncode == 0, out.stderr
+    assert out.stdout.strip() == "LOUD True"
