@@ -445,3 +445,59 @@ def test_iteration_cap_sets_status(tiny):
     hi = np.full(8, 2**31 - 1, np.int32)
     res = oracle.search(ix, wl.queries[:8], lo, hi, 10, 64, max_iters=5)
     assert np.all(res.stats[:, 0] == 5) and np.all(res.status & oracle.ST_ITER_CAP)
+
+
+# ---------------------------------------------------------------------------------------------
+# Alg. 2 main loop (lines 5-18) against a run worked by hand on a 16-vertex index
+# ---------------------------------------------------------------------------------------------
+def _alg2_golden_index():
+    from alg2_golden import load
+    g = load()
+    ix = oracle.OracleIndex(n=g["n"], d=g["d"], d_pad=g["d_pad"], H=g["H"], m=g["m"], n_inv=0, ef_c=0, patience=0,
+                            beta=0.0, gamma=0.0, seed=0, sorted_attr=g["sorted_attr"], rank2id=g["rank2id"],
+                            vectors=g["vectors"], enc=g["enc"])
+    return g, ix
+
+
+def test_alg2_hand_trace_preconditions():
+    """The inputs the hand trace starts from: endpoints, hotspot layers, entry points."""
+    g, ix = _alg2_golden_index()
+    assert oracle.rank_interval(ix.sorted_attr, g["lo"], g["hi"]) == (g["l_q"], g["r_q"])
+    assert list(oracle.hotspot(g["l_q"], g["r_q"], g["H"], g["n"])) == g["hotspot"]
+    eps = [oracle.entry_point(g["seed"], g["l_q"], g["r_q"], j) for j in range(g["epn"])]
+    assert eps == g["entry_points"]
+
+
+@pytest.mark.parametrize("warp", [2, 3, 32])
+def test_alg2_hand_trace(warp):
+    """Sequence of expanded vertices, EN(u) of every expansion, the pool after every merge (read
+    back by stopping the loop after t expansions with k = ef_s), the result and the counters."""
+    g, ix = _alg2_golden_index()
+    lo = np.array([g["lo"]], dtype=np.int32)
+    hi = np.array([g["hi"]], dtype=np.int32)
+    kw = dict(epn=g["epn"], B=g["B"], seed=g["seed"], warp=warp)
+    res = oracle.search(ix, g["query"], lo, hi, g["k"], g["ef_s"], trace_cap=256, **kw)
+    tr = res.trace[0]
+    rec, p = [], 1
+    while p < 1 + tr[0]:
+        cnt = int(tr[p + 1])
+        rec.append((int(tr[p]), [int(v) for v in tr[p + 2:p + 2 + cnt]]))
+        p += 2 + cnt
+    assert rec == [(e["u"], e["en"]) for e in g["exp"]]
+    assert res.ids[0].tolist() == g["result_ids"]
+    assert np.array_equal(res.dists[0], np.sqrt(np.array(g["result_dist2"], dtype=np.float32)))
+    assert res.status[0] == 0
+    assert res.stats[0, 0] == g["stats_expansions"] and res.stats[0, 2] == g["stats_en"]
+    assert res.stats[0, 3] == g["stats_distances"]
+    if warp in (3, 32):
+        assert res.stats[0, 1] == g["stats_rows_chunk%d" % warp]
+    # the pool after t merges: stop after t expansions and return the whole pool
+    for t, e in enumerate(g["exp"], start=1):
+        cut = oracle.search(ix, g["query"], lo, hi, g["ef_s"], g["ef_s"], max_iters=t, **kw)
+        ranks = [r for r, _ in e["pool"]]
+        assert cut.ids[0].tolist() == [int(g["rank2id"][r]) for r in ranks], t
+        assert np.array_equal(cut.dists[0], np.sqrt(np.array([d2 for _, d2 in e["pool"]], dtype=np.float32))), t
+        assert bool(cut.status[0] & oracle.ST_ITER_CAP) == (t < len(g["exp"]))
+    # termination follows ef_s, not k: asking for fewer results does not shorten the run
+    res2 = oracle.search(ix, g["query"], lo, hi, 2, g["ef_s"], **kw)
+    assert res2.stats[0, 0] == g["stats_expansions"] and res2.ids[0].tolist() == g["result_ids"][:2]
