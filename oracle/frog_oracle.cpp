@@ -98,20 +98,24 @@ bool boundary_refinement_invalid(int64_t l_q, int64_t r_q, int h, int64_t N) {
 
 // ---------------------------------------------------------------------------------------------
 // Alg. 3: HotspotLocalization(l_q, r_q, H, N) -> (L_start, L_end).
+// Rule 1 (the descent of Alg. 3 lines 1-12), stated by what it finds rather than how: the walk
+// from the root follows the child that holds the whole range and stops where the range is cut,
+// so L_start is the deepest retained layer at which l_q and r_q still lie in the same segment.
+// Rule 2 (lines 13-22): L_end grows over the following layers while Eq. 6 holds.
 // ---------------------------------------------------------------------------------------------
 void hotspot_localization(int64_t l_q, int64_t r_q, int H, int64_t N, int* L_start, int* L_end) {
-    int64_t L = 0, R = N - 1;
-    int d = 0;
-    while (d < H - 1) {
-        int64_t mid = L + (R - L) / 2;
-        if (r_q <= mid) R = mid;
-        else if (l_q >= mid + 1) L = mid + 1;
-        else break;
-        d = d + 1;
+    int deepest_shared = 0;                       // layer 0 is one segment: it always holds both ends
+    for (int h = 1; h <= H - 1; ++h) {
+        int64_t La, Ra, Lb, Rb;
+        segment_at(N, h, l_q, &La, &Ra);
+        segment_at(N, h, r_q, &Lb, &Rb);
+        if (La != Lb) break;                      // the layer-h segmentation cuts [l_q, r_q]
+        (void)Ra; (void)Rb;
+        deepest_shared = h;
     }
-    *L_start = d;
-    *L_end = d;
-    for (int h = d + 1; h <= H - 1; ++h) {
+    *L_start = deepest_shared;
+    *L_end = deepest_shared;
+    for (int h = deepest_shared + 1; h <= H - 1; ++h) {
         if (boundary_refinement_invalid(l_q, r_q, h, N)) break;
         *L_end = h;
     }

@@ -425,6 +425,41 @@ def test_eager_hash_check_ablation(tiny_runs):
     assert (res.stats[m, 3] / res.stats[m, 0]).mean() >= (base.stats[m, 3] / base.stats[m, 0]).mean()
 
 
+@pytest.mark.parametrize("warp", [16, 32])
+def test_eager_ablation_chunk_by_chunk_replay(tiny_runs, warp):
+    """The eager form depends on the chunk width (a second copy of an id inside one chunk is admitted,
+    takes a slot and fails the insertion).  Alg. 4 takes its chunks inside one layer row (width m = 16
+    here); the CUDA kernel's ablation switch scans 32 entries, i.e. two rows, per chunk.  Both widths
+    are replayed from the recorded sequence of expanded vertices with a plain sequential filter."""
+    wl, ix, _, _, _ = tiny_runs
+    B = 16
+    res = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 48, B=B, eager_hash=True, warp=warp, trace_cap=8192)
+    checked = 0
+    for q in range(wl.nq):
+        if res.status[q] & (oracle.ST_EXACT | oracle.ST_EMPTY):
+            continue
+        l, r = oracle.rank_interval(ix.sorted_attr, int(wl.lo[q]), int(wl.hi[q]))
+        ls, le = oracle.hotspot(l, r, ix.H, ix.n)
+        seen = {oracle.entry_point(0, l, r, j) for j in range(16)}
+        tr = res.trace[q]
+        pos, ln = 1, int(tr[0])
+        while pos < 1 + ln:
+            u, cnt = int(tr[pos]), int(tr[pos + 1])
+            flat = [int(v) for v in np.asarray(ix.enc[u, ls:le + 1]).ravel()]
+            expect = []
+            for c0 in range(0, len(flat), warp):
+                passing = [v for v in flat[c0:c0 + warp] if v != 0xFFFFFFFF and l <= v <= r and v not in seen]
+                take = passing[:B - len(expect)]
+                expect += take
+                seen |= set(take)
+                if len(expect) == B:
+                    break
+            assert [int(x) for x in tr[pos + 2: pos + 2 + cnt]] == expect
+            pos += 2 + cnt
+            checked += 1
+    assert checked > 1000
+
+
 def test_recall_improves_with_beam_and_is_high(tiny_runs):
     wl, ix, gt_ids, _, runs = tiny_runs
     rec = {ef: oracle.recall(res.ids, gt_ids) for ef, res in runs.items()}
