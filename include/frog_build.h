@@ -6,6 +6,7 @@
  * leaves, then per layer the own-child graph neighbours plus a greedy search, Alg. 1, in the
  * sibling's temporary graph; the 2m candidates are RNG-pruned into the parent graph and
  * re-ranked by fusion distance into the layer's ENCs), with the patience rule of Sec. 6.2.2.
+ * Every object works on at most 64 candidates per layer; m <= 32.
  * The search path never calls this; it only reads the file.
  */
 #ifndef FROG_BUILD_H_
@@ -26,8 +27,14 @@ typedef struct {
     float gamma;       /* Eq. 3; <= 0 = 0.5 */
     uint64_t seed;     /* recorded in the header (the build itself is deterministic) */
     int32_t threads;   /* worker threads; 0 = all cores.  The result does not depend on it. */
-    int32_t reserved;
+    int32_t reserved;  /* FROG_BUILD_* switches below, or 0 */
 } frog_build_params_t;
+
+/* Switches (bits of `reserved`, recorded in the file header at byte 68).  The builders add two steps
+ * to the construction of Sec. 6.1; each bit removes one, both together give the section as written. */
+#define FROG_BUILD_NO_REVERSE_EDGES 1   /* candidates are not extended by the sources of incoming edges */
+#define FROG_BUILD_ENC_FUSION_NEAREST 2 /* ENCs = the m fusion-nearest candidates (no RNG rule on them) */
+#define FROG_BUILD_LITERAL 3            /* both */
 
 /* frog_index_build: build the index of n objects and write it to `path`.
  *   vectors  HOST, n x d fp32 row-major, row i = object i

@@ -3,24 +3,38 @@
 // n x H x m ENC array), Sec. 5.2 (fusion distance, Eq. 3), Sec. 6.1 (bottom-up construction:
 // brute-force leaves, then per layer the own-child neighbours plus a greedy search, Alg. 1, in
 // the sibling's temporary vector-distance graph), Sec. 6.2.2 (patience early termination).
+// The CUDA builder (frog_build_gpu.cu) follows the same sentences and writes the same file, bit
+// for bit; this program is its CPU counterpart and the two are compared element by element.
 // Choices where the paper is silent, and two additions:
 //   * ranks by (attribute, object id); H = max(1, ceil(log2 n) + 1 - n_inv);
+//   * vector distance: squared L2 in fp32, rows cut into 4-float groups, group g to partial sum
+//     g mod 8, fused multiply-adds in increasing index, partial sums combined pairwise at distance
+//     4, 2, 1 (the order of the search path).  The distance BETWEEN TWO CANDIDATES used by the RNG
+//     rule is that distance taken over column chunks of 128 floats and summed chunk by chunk (for
+//     d <= 128 it is the same number);
 //   * delta_a = |rank_i - rank_j| / (n - 1); delta_f evaluated in double from sqrt of the fp32
-//     squared distance; ENC rows stored in ascending (delta_f, rank), empty entries at the tail;
-//   * sibling search (Alg. 1): pool width ef_c, entry point = middle rank of the sibling, the m
-//     best of the pool are taken;
-//   * own-child neighbours: every object carries its m nearest (unpruned) of the current segment
-//     upward, next to the pruned graph row used for navigation;
+//     squared distance (delta_a^gamma is sqrt(delta_a) for the default gamma = 0.5, pow otherwise);
+//     orders are (delta_v, rank) and (delta_f, rank); ENC rows stored in ascending delta_f,
+//     empty entries at the tail;
+//   * every object works on at most 64 candidates per layer.  Leaf layer: the 64 nearest other
+//     objects of its leaf (all of them when the leaf has no more than 65).  Inner layers: the m
+//     nearest it already has in its own child segment plus the m best of a greedy search (Alg. 1:
+//     pool width ef_c, entry point = middle rank of the sibling, patience rule of Sec. 6.2.2 with
+//     "improvement" = a new candidate enters the m best, at most 4 ef_c expansions) in the
+//     sibling's temporary graph;
 //   * RNG prune (rule not spelled out in the paper): visit candidates in ascending order, keep c
 //     iff it is closer to u than to every neighbour kept so far, stop at m, back-fill with the
 //     first rejected ones;
-//   * ADDITION 1, reverse edges: the sources of an object's incoming forward edges join its
-//     candidates.  Without them hubs absorb the edges, about a third of the objects get no
-//     incoming edge at the upper layers, the construction searches of the next layer cannot find
-//     them, and search recall saturates near 0.75 on clustered data;
-//   * ADDITION 2, ENC selection: the m ENCs are chosen by the same RNG rule applied in ascending
-//     FUSION distance (the paper keeps the m fusion-nearest); plain top-m gives a k-NN-like
-//     graph that navigates poorly on low-intrinsic-dimension mixtures;
+//   * ADDITION 1, reverse edges (switch FROG_BUILD_NO_REVERSE_EDGES turns it off): a forward graph
+//     row is RNG-selected from the candidates, and the sources of an object's incoming forward
+//     edges join its candidates (the 64 nearest of the union are kept).  Without them hubs absorb
+//     the edges, about a third of the objects get no incoming edge at the upper layers, the
+//     construction searches of the next layer cannot find them, and search recall saturates near
+//     0.75 on clustered data;
+//   * ADDITION 2, ENC selection (switch FROG_BUILD_ENC_FUSION_NEAREST turns it off): the m ENCs
+//     are chosen by the same RNG rule applied in ascending FUSION distance; the paper keeps the m
+//     fusion-nearest, which gives a k-NN-like graph that navigates poorly on low-intrinsic-
+//     dimension mixtures.  With both switches set the builder is the paper's Sec. 6.1 as written;
 //   * the parent graph is written to a second buffer and swapped (the paper overwrites in place);
 //     the result does not depend on the thread count.
 #include "frog_build.h"
@@ -42,20 +56,35 @@ namespace {
 
 constexpr uint32_t BOT = 0xFFFFFFFFu;
 
+constexpr int CAND = 64;          // candidates an object works on per layer
+constexpr int PAIR_CHUNK = 128;   // floats per column chunk of the candidate-to-candidate distance
+
+// squared L2 over d floats (d a multiple of 4): 8 partial sums over 4-float groups, fused
+// multiply-adds in increasing index, combined pairwise at distance 4, 2, 1
 inline float sqdist(const float* a, const float* b, int d) {
-    // eight independent partial sums: vectorisable without re-association
-    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    int i = 0;
-    for (; i + 8 <= d; i += 8)
-        for (int j = 0; j < 8; ++j) {
-            float t = a[i + j] - b[i + j];
-            acc[j] += t * t;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    const int groups = d >> 2;
+    for (int g = 0; g < groups; ++g) {
+        float s = acc[g & 7];
+        for (int e = 0; e < 4; ++e) {
+            const float t = a[4 * g + e] - b[4 * g + e];
+            s = fmaf(t, t, s);
         }
-    for (; i < d; ++i) {
-        float t = a[i] - b[i];
-        acc[i & 7] += t * t;
+        acc[g & 7] = s;
     }
-    return ((acc[0] + acc[4]) + (acc[2] + acc[6])) + ((acc[1] + acc[5]) + (acc[3] + acc[7]));
+    for (int off = 4; off >= 1; off >>= 1) {
+        float nxt[8];
+        for (int t = 0; t < 8; ++t) nxt[t] = acc[t] + acc[t ^ off];
+        for (int t = 0; t < 8; ++t) acc[t] = nxt[t];
+    }
+    return acc[0];
+}
+
+// distance between two candidates (RNG rule): the same, chunk by chunk
+inline float pair_sqdist(const float* a, const float* b, int d) {
+    float s = 0.f;
+    for (int c0 = 0; c0 < d; c0 += PAIR_CHUNK) s += sqdist(a + c0, b + c0, std::min(PAIR_CHUNK, d - c0));
+    return s;
 }
 
 int ceil_log2(int64_t n) {
@@ -119,7 +148,7 @@ struct Searcher {
         pool.push_back(Nb{sqdist(q, V + (int64_t)ep * d, d), ep});
         flag.push_back(0);
         int pat = patience;
-        for (;;) {
+        for (int it = 0; it < 4 * ef_c; ++it) {
             size_t i = 0;
             while (i < pool.size() && flag[i]) ++i;
             if (i >= pool.size()) break;
@@ -157,7 +186,7 @@ void rng_select(const float* V, int d, const Nb* cand, int nc, int m, std::vecto
         bool ok = (int)kept.size() < m;
         if (ok)
             for (const Nb& p : kept)
-                if (!(c.d2 < sqdist(V + (int64_t)c.id * d, V + (int64_t)p.id * d, d))) {
+                if (!(c.d2 < pair_sqdist(V + (int64_t)c.id * d, V + (int64_t)p.id * d, d))) {
                     ok = false;
                     break;
                 }
@@ -174,14 +203,15 @@ inline bool fznb_less(const FzNb& a, const FzNb& b) { return a.f != b.f ? a.f < 
 
 // ENC row: candidates visited in ascending fusion distance (Eq. 3); c is kept iff it is closer
 // (vector distance) to the source than to every ENC kept so far; back-fill in fusion order up to
-// m; the row is stored in ascending fusion distance, empty entries at the tail.
-void select_encs(const float* V, int d, const std::vector<FzNb>& byf, int m, uint32_t* erow) {
+// m; the row is stored in ascending fusion distance, empty entries at the tail.  With
+// `fusion_nearest` the row is simply the m fusion-nearest candidates (the paper's rule).
+void select_encs(const float* V, int d, const std::vector<FzNb>& byf, int m, bool fusion_nearest, uint32_t* erow) {
     std::vector<const FzNb*> kept, pruned;
     for (const FzNb& c : byf) {
         bool ok = (int)kept.size() < m;
-        if (ok)
+        if (ok && !fusion_nearest)
             for (const FzNb* p : kept)
-                if (!(c.nb.d2 < sqdist(V + (int64_t)c.nb.id * d, V + (int64_t)p->nb.id * d, d))) {
+                if (!(c.nb.d2 < pair_sqdist(V + (int64_t)c.nb.id * d, V + (int64_t)p->nb.id * d, d))) {
                     ok = false;
                     break;
                 }
@@ -237,7 +267,7 @@ extern "C" int frog_index_build(const float* vectors, const int32_t* attrs, int6
     if (P.patience == 0) P.patience = 30;
     if (P.beta < 0) P.beta = 0.2f;
     if (P.gamma <= 0) P.gamma = 0.5f;
-    if (P.m < 1 || P.m > 64 || P.ef_c < P.m || P.patience < 1) return 1;
+    if (P.m < 1 || P.m > 32 || P.ef_c < P.m || P.patience < 1) return 1;
     const int m = P.m;
     const int H = frog_retained_depth(n, P.n_inv);
     const int d_pad = (d + 3) / 4 * 4;
@@ -281,61 +311,30 @@ extern "C" int frog_index_build(const float* vectors, const int32_t* attrs, int6
         const double beta = P.beta, gamma = P.gamma;
         const double inv_span = n > 1 ? 1.0 / (double)(n - 1) : 0.0;
         auto fusion = [&](float d2, int64_t ru, int64_t rv) {
-            double da = (double)(ru > rv ? ru - rv : rv - ru) * inv_span;
-            return frog_fusion_distance(std::sqrt((double)d2), da, beta, gamma);
+            const double da = (double)(ru > rv ? ru - rv : rv - ru) * inv_span;
+            const double dv = std::sqrt((double)d2);
+            const double za = gamma == 0.5 ? std::sqrt(da) : std::pow(da, gamma);   // both exact for 0.5
+            return dv * (1.0 - beta * (1.0 - za));
         };
 
-        // ---- leaves (layer H-1): brute force inside each leaf ------------------------------
-        {
-            std::vector<int64_t> starts = layer_starts(n, H - 1);
-#pragma omp parallel
-            {
-                std::vector<Nb> byv, kept, pruned;
-                std::vector<FzNb> byf;
-#pragma omp for schedule(dynamic, 64)
-                for (int64_t u = 0; u < n; ++u) {
-                    size_t s = std::upper_bound(starts.begin(), starts.end(), u) - starts.begin() - 1;
-                    int64_t L = starts[s], R = starts[s + 1] - 1;
-                    byv.clear();
-                    byf.clear();
-                    for (int64_t v = L; v <= R; ++v) {
-                        if (v == u) continue;
-                        byv.push_back(Nb{sqdist(V + u * d_pad, V + v * d_pad, d_pad), (uint32_t)v});
-                    }
-                    std::sort(byv.begin(), byv.end(), nb_less);
-                    for (const Nb& c : byv) byf.push_back(FzNb{fusion(c.d2, u, c.id), c});
-                    std::sort(byf.begin(), byf.end(), fznb_less);
-                    rng_select(V, d_pad, byv.data(), (int)byv.size(), m, kept, pruned);
-                    for (int j = 0; j < m; ++j) {
-                        pg_cur[u * m + j] = j < (int)kept.size() ? kept[j].id : BOT;
-                        ann_cur[u * m + j] = j < (int)byv.size() ? byv[j].id : BOT;
-                        pd_cur[u * m + j] = j < (int)byv.size() ? byv[j].d2 : 0.f;
-                    }
-                    select_encs(V, d_pad, byf, m, enc + ((int64_t)u * H + (H - 1)) * m);
-                }
-            }
-        }
-
-        // ---- inductive step, layers H-2 .. 0 -----------------------------------------------
-        // Per layer: (1) every object collects 2m vector-distance candidates -- the m nearest it
-        // already has in its own child segment plus the m found by a greedy search (Alg. 1) in the
-        // sibling's temporary graph; (2) a forward graph row is RNG-pruned from them; (3) each
-        // object adds the sources of its incoming forward edges to its candidates (without them a
-        // third of the objects end up with no incoming edge and can never be found again, neither
-        // by the next layer's construction searches nor at query time) and derives from this pool
-        // its nearest list, the parent's temporary graph row, and the layer's ENCs.
+        // ---- layers H-1 .. 0 ----------------------------------------------------------------
+        // Per layer: (1) every object collects its candidates in ascending (delta_v, rank) -- leaf
+        // layer: the nearest CAND other objects of its leaf; inner layers: the m nearest it already
+        // has in its own child segment plus the m found by a greedy search (Alg. 1) in the sibling's
+        // temporary graph; (2) a forward graph row is RNG-selected from them; (3) each object adds
+        // the sources of its incoming forward edges to its candidates (nearest CAND of the union)
+        // and derives from this pool its nearest list, the parent's temporary graph row, and the
+        // layer's ENCs.
         std::vector<Searcher> searchers(nthreads);
-        const int C = 2 * m;   // candidates per object
-        std::unique_ptr<Nb[]> c1p;
-        std::unique_ptr<uint32_t[]> pgF;
-        if (H > 1) {
+        if (H > 1)
             for (auto& s : searchers) s.init(n, P.ef_c);
-            c1p.reset(new Nb[(size_t)n * C]);
-            pgF.reset(new uint32_t[(size_t)n * m]);
-        }
+        std::unique_ptr<Nb[]> c1p(new Nb[(size_t)n * CAND]);
+        std::unique_ptr<uint32_t[]> pgF(new uint32_t[(size_t)n * m]);
         Nb* c1 = c1p.get();
         uint32_t* pg_fwd = pgF.get();
-        for (int h = H - 2; h >= 0; --h) {
+        const bool reverse_edges = !(P.reserved & FROG_BUILD_NO_REVERSE_EDGES);
+        const bool fusion_nearest = (P.reserved & FROG_BUILD_ENC_FUSION_NEAREST) != 0;
+        for (int h = H - 1; h >= 0; --h) {
             std::vector<int64_t> starts = layer_starts(n, h);
             // (1) + (2)
 #pragma omp parallel
@@ -350,31 +349,37 @@ extern "C" int frog_index_build(const float* vectors, const int32_t* attrs, int6
                 for (int64_t u = 0; u < n; ++u) {
                     size_t s = std::upper_bound(starts.begin(), starts.end(), u) - starts.begin() - 1;
                     int64_t L = starts[s], R = starts[s + 1] - 1;
-                    int64_t mid = L + (R - L) / 2;
-                    int64_t sL, sR;   // sibling child segment
-                    if (u <= mid) { sL = mid + 1; sR = R; } else { sL = L; sR = mid; }
                     cand.clear();
-                    for (int j = 0; j < m; ++j)
-                        if (ann_cur[u * m + j] != BOT) cand.push_back(Nb{pd_cur[u * m + j], ann_cur[u * m + j]});
-                    if (sL <= sR) {
-                        uint32_t ep = (uint32_t)(sL + (sR - sL) / 2);
-                        S.run(V, d_pad, pg_cur, m, V + u * d_pad, ep, P.ef_c, P.patience, m);
-                        size_t take = std::min<size_t>(m, S.pool.size());
-                        for (size_t j = 0; j < take; ++j) cand.push_back(S.pool[j]);
+                    if (h == H - 1) {
+                        for (int64_t v = L; v <= R; ++v)
+                            if (v != u) cand.push_back(Nb{sqdist(V + u * d_pad, V + v * d_pad, d_pad), (uint32_t)v});
+                    } else {
+                        int64_t mid = L + (R - L) / 2;
+                        int64_t sL, sR;   // sibling child segment
+                        if (u <= mid) { sL = mid + 1; sR = R; } else { sL = L; sR = mid; }
+                        for (int j = 0; j < m; ++j)
+                            if (ann_cur[u * m + j] != BOT) cand.push_back(Nb{pd_cur[u * m + j], ann_cur[u * m + j]});
+                        if (sL <= sR) {
+                            uint32_t ep = (uint32_t)(sL + (sR - sL) / 2);
+                            S.run(V, d_pad, pg_cur, m, V + u * d_pad, ep, P.ef_c, P.patience, m);
+                            size_t take = std::min<size_t>(m, S.pool.size());
+                            for (size_t j = 0; j < take; ++j) cand.push_back(S.pool[j]);
+                        }
                     }
                     std::sort(cand.begin(), cand.end(), nb_less);
-                    for (int j = 0; j < C; ++j) c1[u * C + j] = j < (int)cand.size() ? cand[j] : Nb{0.f, BOT};
+                    if ((int)cand.size() > CAND) cand.resize(CAND);
+                    for (int j = 0; j < CAND; ++j) c1[u * CAND + j] = j < (int)cand.size() ? cand[j] : Nb{0.f, BOT};
                     rng_select(V, d_pad, cand.data(), (int)cand.size(), m, kept, pruned);
                     for (int j = 0; j < m; ++j) pg_fwd[u * m + j] = j < (int)kept.size() ? kept[j].id : BOT;
                 }
             }
             // reverse edges of the forward graph, grouped by target, sources ascending
             std::vector<uint32_t> rev_off((size_t)n + 1, 0), rev_src;
-            for (int64_t e = 0; e < n * m; ++e)
-                if (pg_fwd[e] != BOT) ++rev_off[(size_t)pg_fwd[e] + 1];
-            for (int64_t v = 0; v < n; ++v) rev_off[v + 1] += rev_off[v];
-            rev_src.resize(rev_off[n]);
-            {
+            if (reverse_edges) {
+                for (int64_t e = 0; e < n * m; ++e)
+                    if (pg_fwd[e] != BOT) ++rev_off[(size_t)pg_fwd[e] + 1];
+                for (int64_t v = 0; v < n; ++v) rev_off[v + 1] += rev_off[v];
+                rev_src.resize(rev_off[n]);
                 std::vector<uint32_t> cur(rev_off.begin(), rev_off.end() - 1);
                 for (int64_t u = 0; u < n; ++u)
                     for (int j = 0; j < m; ++j) {
@@ -389,9 +394,9 @@ extern "C" int frog_index_build(const float* vectors, const int32_t* attrs, int6
                 std::vector<FzNb> byf;
 #pragma omp for schedule(dynamic, 64)
                 for (int64_t u = 0; u < n; ++u) {
-                    const Nb* cand = c1 + u * C;
+                    const Nb* cand = c1 + u * CAND;
                     pool.clear();
-                    for (int j = 0; j < C && cand[j].id != BOT; ++j) pool.push_back(cand[j]);
+                    for (int j = 0; j < CAND && cand[j].id != BOT; ++j) pool.push_back(cand[j]);
                     const size_t base = pool.size();
                     for (uint32_t e = rev_off[u]; e < rev_off[u + 1]; ++e) {
                         uint32_t v = rev_src[e];
@@ -401,7 +406,7 @@ extern "C" int frog_index_build(const float* vectors, const int32_t* attrs, int6
                         if (!known) pool.push_back(Nb{sqdist(V + u * d_pad, V + (int64_t)v * d_pad, d_pad), v});
                     }
                     std::sort(pool.begin(), pool.end(), nb_less);
-                    if ((int)pool.size() > 2 * C) pool.resize(2 * C);
+                    if ((int)pool.size() > CAND) pool.resize(CAND);
                     const int np = (int)pool.size();
                     for (int j = 0; j < m; ++j) {
                         ann_nxt[u * m + j] = j < np ? pool[j].id : BOT;
@@ -413,7 +418,7 @@ extern "C" int frog_index_build(const float* vectors, const int32_t* attrs, int6
                     byf.clear();
                     for (int ci = 0; ci < np; ++ci) byf.push_back(FzNb{fusion(pool[ci].d2, u, pool[ci].id), pool[ci]});
                     std::sort(byf.begin(), byf.end(), fznb_less);
-                    select_encs(V, d_pad, byf, m, enc + ((int64_t)u * H + h) * m);
+                    select_encs(V, d_pad, byf, m, fusion_nearest, enc + ((int64_t)u * H + h) * m);
                 }
             }
             std::swap(pg_cur, pg_nxt);
@@ -435,6 +440,8 @@ extern "C" int frog_index_build(const float* vectors, const int32_t* attrs, int6
         std::memcpy(hdr + 56, &P.seed, 8);
         uint32_t bot = BOT;
         std::memcpy(hdr + 64, &bot, 4);
+        uint32_t flags = (uint32_t)P.reserved & (FROG_BUILD_NO_REVERSE_EDGES | FROG_BUILD_ENC_FUSION_NEAREST);
+        std::memcpy(hdr + 68, &flags, 4);
         uint64_t off_attr = 256;
         uint64_t off_r2i = align128(off_attr + (uint64_t)n * 4);
         uint64_t off_vec = align128(off_r2i + (uint64_t)n * 4);

@@ -61,7 +61,16 @@ struct BuildArgs {
     uint32_t* bitmap;        // visited slabs of the sibling searches
     size_t bitmap_words;
     int h;                   // layer under construction
+    int fusion_nearest;      // ENCs = the m fusion-nearest candidates (no RNG rule on them)
+    int wait_limit;          // polls a wait on a bulk copy may take before giving up
+    int skip_copies;         // test hook: expect the bytes but issue no copy, so that every wait runs out
+    uint32_t* fail;          // set to 1 when a wait gave up: the build is not valid
 };
+
+// bounded wait on the bulk copies of a pass; records a give-up in *fail
+__device__ __forceinline__ void wait_copies(const BuildArgs& A, uint64_t* bar, uint32_t phase) {
+    if (!mbar_wait_limit(bar, phase, A.wait_limit)) *A.fail = 1u;
+}
 
 // shared-memory slice of one warp in the candidate / search / pool kernels
 struct BWarp {
@@ -97,7 +106,8 @@ __device__ __forceinline__ uint64_t cand_keys(const BuildArgs& A, const BWarp& W
     const uint32_t id = lane < ns ? W.cand[lane] : 0u;
     float d2 = 0.f;
     bool ok = true;
-    if (ns > 0) d2 = staged_dist2<8>(A.V, A.d_pad, W.q, W.stage, W.bar, phase, ok, id, ns, lane);
+    if (ns > 0) d2 = staged_dist2<8>(A.V, A.d_pad, W.q, W.stage, W.bar, phase, ok, id, ns, lane, A.wait_limit, !A.skip_copies);
+    if (!ok) *A.fail = 1u;
     return lane < ns ? make_key(d2, id, flag) : KEY_EMPTY;
 }
 
@@ -335,17 +345,17 @@ select_kernel(const BuildArgs A) {
         for (int c0 = 0; c0 < row_bytes; c0 += STAGE_CHUNK) {
             const int cbytes = min(STAGE_CHUNK, row_bytes - c0);
             __syncwarp();
-            if (lane == 0) mbar_expect_tx(S.bar, (uint32_t)(K * cbytes));
+            if (lane == 0 && !A.skip_copies) mbar_expect_tx(S.bar, (uint32_t)(K * cbytes));
             __syncwarp();
 #pragma unroll
             for (int rr = 0; rr < 2; ++rr) {
                 const int r = lane + 32 * rr;
-                if (r < K)
+                if (r < K && !A.skip_copies)
                     tma_load_1d(reinterpret_cast<char*>(S.stage) + (size_t)r * STAGE_CHUNK,
                                 reinterpret_cast<const char*>(A.V) + (size_t)key_rank(S.keys[r]) * row_bytes + c0,
                                 (uint32_t)cbytes, S.bar);
             }
-            mbar_wait(S.bar, phase);
+            wait_copies(A, S.bar, phase);
             phase ^= 1u;
             const int g_n = cbytes >> 4;
             for (int i = 0; i + 1 < K; ++i) {
@@ -392,7 +402,8 @@ select_kernel(const BuildArgs A) {
                 if (i < K) {
                     const double dv = sqrt((double)key_dist2(S.keys[i]));
                     const double da = fabs((double)u - (double)key_rank(S.keys[i])) * A.inv_span;
-                    S.fus[i] = dv * (1.0 - A.beta * (1.0 - pow(da, A.gamma)));
+                    const double za = A.gamma == 0.5 ? sqrt(da) : pow(da, A.gamma);   // sqrt is exact on both builders
+                    S.fus[i] = dv * (1.0 - A.beta * (1.0 - za));
                 }
             }
             __syncwarp();
@@ -411,7 +422,13 @@ select_kernel(const BuildArgs A) {
                 }
             }
             __syncwarp();
-            nk = rng_rule(S, K, A.m, lane);
+            if (A.fusion_nearest) {
+                nk = min(K, A.m);                              // the paper's rule: the m fusion-nearest
+                if (lane < nk) S.kept[lane] = S.ord[lane];
+                __syncwarp();
+            } else {
+                nk = rng_rule(S, K, A.m, lane);
+            }
             // store the kept candidates in ascending fusion distance (their position in ord)
             uint32_t* erow = A.enc + ((size_t)u * A.H + A.h) * A.m;
             int kpos = 0x7FFFFFFF;
@@ -533,8 +550,15 @@ extern "C" int frog_index_build_gpu(const float* vectors, const int32_t* attrs, 
         (rc = buf.alloc(&pgA, nm)) || (rc = buf.alloc(&pgB, nm)) || (rc = buf.alloc(&pdA, nm)) ||
         (rc = buf.alloc(&pdB, nm)) || (rc = buf.alloc(&A.fwd, nm)) || (rc = buf.alloc(&A.enc, nm * H)) ||
         (rc = buf.alloc(&A.rev_cnt, (size_t)n + 1)) || (rc = buf.alloc(&A.rev_off, (size_t)n + 1)) ||
-        (rc = buf.alloc(&A.rev_cur, (size_t)n)) || (rc = buf.alloc(&A.rev_src, nm)))
+        (rc = buf.alloc(&A.rev_cur, (size_t)n)) || (rc = buf.alloc(&A.rev_src, nm)) || (rc = buf.alloc(&A.fail, 1)))
         return rc;
+    FROG_CUDA_TRY(cudaMemset(A.fail, 0, sizeof(uint32_t)));
+    const bool reverse_edges = !(P.reserved & FROG_BUILD_NO_REVERSE_EDGES);
+    A.fusion_nearest = (P.reserved & FROG_BUILD_ENC_FUSION_NEAREST) ? 1 : 0;
+    // test hook (bits 16..31 of `reserved`): a nonzero value v makes every wait give up after v polls
+    // and neither arms the barriers nor issues a copy, so that the give-up path runs with nothing in flight
+    A.wait_limit = (P.reserved >> 16) ? (P.reserved >> 16) : (1 << 22);
+    A.skip_copies = (P.reserved >> 16) ? 1 : 0;
     FROG_CUDA_TRY(cudaMemcpy(dV, Vh.get(), (size_t)n * d_pad * 4, cudaMemcpyHostToDevice));
     A.V = dV;
     A.n = n; A.d_pad = d_pad; A.H = H; A.m = m; A.ef_c = P.ef_c; A.patience = P.patience;
@@ -578,9 +602,13 @@ extern "C" int frog_index_build_gpu(const float* vectors, const int32_t* attrs, 
         select_kernel<false><<<g_sel0, 32, SEL_BYTES>>>(A);
         FROG_CUDA_TRY(cudaMemsetAsync(A.rev_cnt, 0, ((size_t)n + 1) * 4));
         FROG_CUDA_TRY(cudaMemsetAsync(A.rev_cur, 0, (size_t)n * 4));
-        rev_count_kernel<<<eg, eb>>>(A.fwd, edges, A.rev_cnt);
-        thrust::exclusive_scan(thrust::device, A.rev_cnt, A.rev_cnt + n + 1, A.rev_off);
-        rev_fill_kernel<<<eg, eb>>>(A.fwd, edges, m, A.rev_off, A.rev_cur, A.rev_src);
+        if (reverse_edges) {
+            rev_count_kernel<<<eg, eb>>>(A.fwd, edges, A.rev_cnt);
+            thrust::exclusive_scan(thrust::device, A.rev_cnt, A.rev_cnt + n + 1, A.rev_off);
+            rev_fill_kernel<<<eg, eb>>>(A.fwd, edges, m, A.rev_off, A.rev_cur, A.rev_src);
+        } else {
+            FROG_CUDA_TRY(cudaMemsetAsync(A.rev_off, 0, ((size_t)n + 1) * 4));      // no incoming sources
+        }
         pool_kernel<<<g_pool, BWARPS * 32, smem_plain>>>(A);
         select_kernel<true><<<g_sel1, 32, SEL_BYTES>>>(A);
         FROG_CUDA_TRY(cudaGetLastError());
@@ -589,6 +617,11 @@ extern "C" int frog_index_build_gpu(const float* vectors, const int32_t* attrs, 
         std::swap(A.pg_cur, A.pg_nxt);
     }
     FROG_CUDA_TRY(cudaDeviceSynchronize());
+    {
+        uint32_t failed = 0;
+        FROG_CUDA_TRY(cudaMemcpy(&failed, A.fail, sizeof(failed), cudaMemcpyDeviceToHost));
+        if (failed) return FROG_ERR_CUDA;      // a bulk copy never completed: no file is written
+    }
 
     std::unique_ptr<uint32_t[]> ench(new (std::nothrow) uint32_t[nm * H]);
     if (!ench) return FROG_ERR_NOMEM;
@@ -608,6 +641,8 @@ extern "C" int frog_index_build_gpu(const float* vectors, const int32_t* attrs, 
     std::memcpy(hdr + 56, &P.seed, 8);
     const uint32_t bot = BOT;
     std::memcpy(hdr + 64, &bot, 4);
+    const uint32_t flags = (uint32_t)P.reserved & (FROG_BUILD_NO_REVERSE_EDGES | FROG_BUILD_ENC_FUSION_NEAREST);
+    std::memcpy(hdr + 68, &flags, 4);
     const uint64_t off_attr = 256, off_r2i = align128(off_attr + nn * 4), off_vec = align128(off_r2i + nn * 4),
                    off_enc = align128(off_vec + nn * d_pad * 4), total = off_enc + nn * H * m * 4;
     const uint64_t offs[5] = {off_attr, off_r2i, off_vec, off_enc, total};
