@@ -70,7 +70,9 @@ typedef struct {
     int32_t visited;    /* FROG_VISITED_*: where the visited set lives */
     int32_t storage;    /* FROG_STORAGE_*: which copy of the vectors the gather reads */
     int32_t debug_flags;/* bit 0: with `trace`, record per-phase cycle counts instead of EN lists;
-                           bit 1: process queries in input order (no heaviest-first planning pass) */
+                           bit 1: process queries in input order (no heaviest-first planning pass);
+                           bit 2: use the general kernel where a kernel specialised for the row size exists
+                                  (same results; for comparing the two) */
     int32_t exact_below;/* ranges holding at most max(beam_width, exact_below) objects are answered by
                            scanning their contiguous rank slab (exact, status FROG_ST_EXACT) instead of
                            the graph search; 0 = default: only ranges that fit the pool.  Not in the
@@ -101,7 +103,8 @@ typedef struct {
 #define FROG_ST_ITER_CAP 4u  /* expansion cap hit; the current pool was returned */
 #define FROG_ST_SHORT 8u     /* fewer than k results; tail is padding */
 #define FROG_ST_COPY_TIMEOUT 32u /* a bulk copy into shared memory did not complete within the kernel's
-                                    polling limit; the row's results are not valid (never expected) */
+                                    polling limit; the row is written as padding (-1, +inf), with
+                                    FROG_ST_SHORT set as well (never expected) */
 #define FROG_ST_FORGOT 16u   /* the visited table overflowed and dropped entries: some distances were
                                 evaluated twice; the results are unaffected */
 

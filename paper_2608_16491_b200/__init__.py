@@ -114,16 +114,20 @@ def retained_depth(n: int, n_inv: int) -> int:
     return int(_build_lib().frog_retained_depth(n, n_inv))
 
 
+BUILD_NO_REVERSE_EDGES, BUILD_ENC_FUSION_NEAREST, BUILD_LITERAL = 1, 2, 3
+
+
 def build_index(vectors: np.ndarray, attrs: np.ndarray, path: str, m: int = 0, ef_c: int = 0,
                 n_inv: int = -1, patience: int = 0, beta: float = -1.0, gamma: float = 0.0,
-                seed: int = 0, threads: int = 0) -> None:
-    """Build the FROG index of (vectors, attrs) on the host and write it to ``path``."""
+                seed: int = 0, threads: int = 0, flags: int = 0) -> None:
+    """Build the FROG index of (vectors, attrs) on the host and write it to ``path``.
+    ``flags``: BUILD_* switches (BUILD_LITERAL = the construction of Sec. 6.1 as written)."""
     v = np.ascontiguousarray(vectors, dtype=np.float32)
     a = np.ascontiguousarray(attrs, dtype=np.int32)
     if v.ndim != 2 or a.shape != (v.shape[0],):
         raise ValueError("vectors must be [n, d] and attrs [n]")
     p = BuildParams(m=m, ef_c=ef_c, n_inv=n_inv, patience=patience, beta=beta, gamma=gamma,
-                    seed=seed, threads=threads, reserved=0)
+                    seed=seed, threads=threads, reserved=flags)
     rc = _build_lib().frog_index_build(v.ctypes.data_as(_vp), a.ctypes.data_as(_vp),
                                        C.c_int64(v.shape[0]), C.c_int32(v.shape[1]), C.byref(p),
                                        path.encode())
@@ -133,14 +137,15 @@ def build_index(vectors: np.ndarray, attrs: np.ndarray, path: str, m: int = 0, e
 
 def build_index_gpu(vectors: np.ndarray, attrs: np.ndarray, path: str, device: int = 0, m: int = 0,
                     ef_c: int = 0, n_inv: int = -1, patience: int = 0, beta: float = -1.0,
-                    gamma: float = 0.0, seed: int = 0) -> None:
-    """Build the FROG index of (vectors, attrs) with the CUDA builder and write it to ``path``."""
+                    gamma: float = 0.0, seed: int = 0, flags: int = 0) -> None:
+    """Build the FROG index of (vectors, attrs) with the CUDA builder and write it to ``path``
+    (the same file the host builder writes).  ``flags``: BUILD_* switches."""
     v = np.ascontiguousarray(vectors, dtype=np.float32)
     a = np.ascontiguousarray(attrs, dtype=np.int32)
     if v.ndim != 2 or a.shape != (v.shape[0],):
         raise ValueError("vectors must be [n, d] and attrs [n]")
     p = BuildParams(m=m, ef_c=ef_c, n_inv=n_inv, patience=patience, beta=beta, gamma=gamma,
-                    seed=seed, threads=0, reserved=0)
+                    seed=seed, threads=0, reserved=flags)
     rc = _lib.frog_index_build_gpu(v.ctypes.data_as(_vp), a.ctypes.data_as(_vp), C.c_int64(v.shape[0]),
                                    C.c_int32(v.shape[1]), C.byref(p), C.c_int(device), path.encode())
     if rc != 0:

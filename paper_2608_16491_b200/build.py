@@ -18,7 +18,7 @@ INCLUDE = os.path.join(ROOT, "include")
 LIB_SEARCH = os.path.join(HERE, "libfrog.so")
 LIB_BUILD = os.path.join(HERE, "libfrog_build.so")
 
-CUDA_SOURCES = ["frog_index.cu", "frog_search.cu", "frog_exact.cu", "frog_build_gpu.cu"]
+CUDA_SOURCES = ["frog_index.cu", "frog_search.cu", "frog_search_lean.cu", "frog_exact.cu", "frog_build_gpu.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--fmad=false", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
@@ -48,17 +48,42 @@ def build_builder(force: bool = False, verbose: bool = False) -> str:
 
 
 def build_search(force: bool = False, verbose: bool = False) -> str:
-    srcs = [os.path.join(CSRC, s) for s in CUDA_SOURCES]
-    if force or _newer(LIB_SEARCH, srcs + _headers()):
-        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + ["-shared", "-I", INCLUDE, "-I", CSRC, "-o", LIB_SEARCH] + srcs
+    """Compile every .cu file to an object of its own (in parallel, only those older than their
+    sources or any header) and link them into libfrog.so."""
+    from concurrent.futures import ThreadPoolExecutor
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    objdir = os.path.join(HERE, "build")
+    os.makedirs(objdir, exist_ok=True)
+    heads = _headers()
+    jobs = []
+    for name in CUDA_SOURCES:
+        src = os.path.join(CSRC, name)
+        obj = os.path.join(objdir, name.replace(".cu", ".o"))
+        if force or _newer(obj, [src] + heads):
+            jobs.append((name, [nvcc] + NVCC_FLAGS + ["-c", "-I", INCLUDE, "-I", CSRC, "-o", obj, src]))
+
+    def run(job):
+        name, cmd = job
         if verbose:
             print(" ".join(cmd))
         out = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
-        if verbose or out.returncode != 0:
-            print(out.stdout)
-        if out.returncode != 0:
-            raise RuntimeError("nvcc failed")
+        return name, out.returncode, out.stdout
+
+    failed = []
+    with ThreadPoolExecutor(max_workers=max(1, len(jobs))) as ex:
+        for name, rc, text in ex.map(run, jobs):
+            if verbose or rc != 0:
+                print(text)
+            if rc != 0:
+                failed.append(name)
+    if failed:
+        raise RuntimeError("nvcc failed on " + ", ".join(failed))
+    objs = [os.path.join(objdir, n.replace(".cu", ".o")) for n in CUDA_SOURCES]
+    if jobs or force or _newer(LIB_SEARCH, objs):
+        cmd = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_SEARCH] + objs
+        if verbose:
+            print(" ".join(cmd))
+        subprocess.check_call(cmd)
     return LIB_SEARCH
 
 

@@ -266,6 +266,18 @@ __device__ __forceinline__ void tma_load_1d_l2(void* dst_smem, const void* src_g
 // Wait for the phase of parity `phase`; bounded: gives up after 2^22 polls and reports false (the
 // caller flags the query instead of hanging the GPU).  try_wait already parks the thread for a
 // hardware-chosen interval per poll; passing an explicit suspend-time hint measured 7 % slower.
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t phase, int limit) {
+    const uint32_t addr = smem_u32(bar);
+    for (int it = 0; it < limit; ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(addr), "r"(phase) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t phase) {
     const uint32_t addr = smem_u32(bar);
     for (int it = 0; it < (1 << 22); ++it) {
@@ -295,7 +307,8 @@ constexpr int STAGE_CHUNK = 512;     // bytes of one row in flight per pass
 template <int STAGE_ROWS>
 __device__ __forceinline__ float staged_dist2(const float* __restrict__ vectors, int d_pad, const float4* qs,
                                               float4* stage, uint64_t* bar, uint32_t& phase, bool& ok,
-                                              uint32_t my_rank, int ns, int lane) {
+                                              uint32_t my_rank, int ns, int lane, int wait_limit = 1 << 22,
+                                              bool issue_copies = true) {
     static_assert(STAGE_ROWS == 8 || STAGE_ROWS == 12 || STAGE_ROWS == 16, "rows per pass");
     const int team = lane >> 3, sub = lane & 7;
     const int row_bytes = d_pad * 4;
@@ -313,11 +326,11 @@ __device__ __forceinline__ float staged_dist2(const float* __restrict__ vectors,
         for (int c0 = 0; c0 < row_bytes; c0 += STAGE_CHUNK) {
             const int cbytes = min(STAGE_CHUNK, row_bytes - c0);
             __syncwarp();                                   // every lane is done reading the stage buffer
-            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(nrows * cbytes));
+            if (lane == 0 && issue_copies) mbar_expect_tx(bar, (uint32_t)(nrows * cbytes));
             __syncwarp();
-            if (lane < nrows)
+            if (lane < nrows && issue_copies)
                 tma_load_1d(reinterpret_cast<char*>(stage) + lane * STAGE_CHUNK, src_row + c0, (uint32_t)cbytes, bar);
-            ok = mbar_wait(bar, phase) && ok;
+            ok = mbar_wait_limit(bar, phase, wait_limit) && ok;
             phase ^= 1u;
             const int g_lo = c0 >> 4, g_n = cbytes >> 4;    // 4-float groups of this chunk
 #pragma unroll
@@ -604,6 +617,33 @@ __device__ __forceinline__ uint64_t warp_min_key(uint64_t key) {
     const uint32_t mhi = __reduce_min_sync(FULL, hi);
     const uint32_t mlo = __reduce_min_sync(FULL, hi == mhi ? lo : 0xFFFFFFFFu);
     return ((uint64_t)mhi << 32) | mlo;
+}
+
+// entry point j of a query range: stateless mixer of (seed, l_q, r_q, j), top 32 bits scaled
+// into [0, w) by a multiply-high (Alg. 2 line 3: uniform sample from [l_q, r_q])
+__device__ __forceinline__ uint32_t entry_point(unsigned long long seed, uint32_t l_q, uint32_t r_q, int j) {
+    unsigned long long x = seed ^ ((unsigned long long)l_q * 0x9E3779B97F4A7C15ull)
+                                ^ ((unsigned long long)r_q * 0xC2B2AE3D27D4EB4Full)
+                                ^ ((unsigned long long)(j + 1) * 0x165667B19E3779F9ull);
+    x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
+    x ^= x >> 27; x *= 0x94D049BB133111EBull;
+    x ^= x >> 31;
+    unsigned long long w = (unsigned long long)(r_q - l_q) + 1ull;
+    return l_q + (uint32_t)(((x >> 32) * w) >> 32);
+}
+
+// Ranges covering at least this many slab words (262,144 objects) log the ranks they evaluate and
+// zero only those words afterwards; narrower ones zero the words of the range (<= 32 KB).
+constexpr int SPARSE_MIN_WORDS = 8192;
+
+// Append the ns <= 64 ranks of cand[] (the vertices whose visited bit this query has just set) to the
+// warp's log.  Returns the new length, or -1 once the log is full: the query then falls back to zeroing
+// the words of its whole range.
+__device__ __forceinline__ int log_ranks(uint32_t* log, int cap, int n_logged, const uint32_t* cand, int ns, int lane) {
+    if (n_logged + ns > cap) return -1;
+    if (lane < ns) __stcg(log + n_logged + lane, cand[lane]);
+    if (lane + 32 < ns) __stcg(log + n_logged + lane + 32, cand[lane + 32]);
+    return n_logged + ns;
 }
 
 }  // namespace frogdev

@@ -1,7 +1,9 @@
 // frog_exact_search: exact filtered kNN (paper Def. 2) by scanning each query's contiguous rank
 // slab (Sec. 4).  One CTA per query; each warp streams batches of 16 consecutive rows through the
 // same distance routine the beam search uses, keeps its own sorted top-k in shared memory, and
-// warp 0 merges the per-warp lists at the end.  Ordering: (squared distance, rank) ascending.
+// warp 0 merges the per-warp lists at the end.  Ordering: (squared distance, original object id)
+// ascending, the total order of Def. 2's tie rule (objects with equal attributes are ranked by id, so
+// this differs from rank order only between equidistant objects with different attributes).
 #include "frog_device.cuh"
 #include "frog_internal.h"
 
@@ -52,7 +54,8 @@ frog_exact_kernel(const ExactArgs A) {
         const int cnt = min(16, w - b0);
         const uint32_t rank = (uint32_t)(l_q + b0 + (lane & 15));
         float d2 = batch_dist2<4>(A.vectors, A.d_pad, qs, rank, cnt, lane);
-        uint64_t key = lane < cnt ? make_key(d2, rank, 1u) : KEY_EMPTY;
+        uint64_t key = KEY_EMPTY;
+        if (lane < cnt) key = make_key(d2, (uint32_t)__ldg(A.rank2id + rank), 1u);   // keyed by object id
         // (merge_batch itself rejects candidates not better than the current k-th best)
         merge_batch<EPL>(pool, key, A.k, lane);
     }
@@ -71,7 +74,7 @@ frog_exact_kernel(const ExactArgs A) {
             int32_t oid = -1;
             float dist = __int_as_float(0x7F800000);
             if (key != KEY_EMPTY) {
-                oid = __ldg(A.rank2id + key_rank(key));
+                oid = (int32_t)key_rank(key);
                 dist = __fsqrt_rn(key_dist2(key));
             }
             A.out_ids[(size_t)q * A.k + j] = oid;

@@ -13,7 +13,7 @@
 // launch that used the set.
 struct FrogScratch {
     unsigned int* d_work = nullptr;  // 1 KB
-    uint32_t* d_bitmap = nullptr;    // bitmap_slots x words per slot
+    uint32_t* d_bitmap = nullptr;    // bitmap_slots x (words of visited bits + log of evaluated ranks)
     size_t bitmap_slots = 0;
     int32_t* d_plan = nullptr;       // per query: rank interval (2 ints) and processing order (1 int)
     size_t plan_queries = 0;
@@ -69,7 +69,11 @@ struct FrogSearchArgs {
     int trace_cap;
     unsigned int* work_counter;
     uint32_t* bitmap;          // visited slabs, or null when the shared-memory table is used
-    size_t bitmap_words;       // words per slab
+    size_t bitmap_words;       // words of visited bits per slab
+    size_t slab_stride;        // words from one warp's slab to the next (bits, then the log of evaluated ranks)
+    int log_cap;               // entries of the per-warp log of evaluated ranks that follows the bits (0: none)
+    int slab_clean;            // nonzero: every slab is all-zero between queries (the kernel restores that
+                               // when a query ends); zero: a query clears the words of its range before use
     const int2* ranges;        // precomputed [l_q, r_q] per query, or null: computed in the kernel
     const int32_t* order;      // processing order (heaviest first), or null: input order
     const void* rows;          // gather source: fp32 vectors, or their fp16 copy
@@ -80,7 +84,11 @@ struct FrogSearchArgs {
     alignas(64) CUtensorMap tmap;
 };
 
+typedef void (*frog_kernel_fn)(const FrogSearchArgs);
+
 namespace froghost {
+// frog_search_lean.cu: the trimmed kernel for 384- and 512-byte fp32 rows (null: shape not covered)
+frog_kernel_fn lean_kernel(int ef_s, int row_bytes, size_t* smem_per_warp, int* warps_per_cta);
 void set_cuda_error(cudaError_t e);
 int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in, frog_params_t* out);
 bool make_row_tensor_map(const void* base, bool f16, int row_elems, size_t row_bytes, size_t n, CUtensorMap* out);

@@ -9,8 +9,11 @@
 //
 // Visited set (the hashCheck of Alg. 2 line 12), two interchangeable forms:
 //   * BITMAP: one bit per rank in a per-warp slab of global scratch memory, test-and-set with a
-//     single atomicOr (exact, no probing, no shared memory; the warp clears the words covering
-//     [l_q, r_q] when it starts a query; the slab stays L2-resident while the query runs);
+//     single atomicOr (exact, no probing, no shared memory; the slab stays L2-resident while the
+//     query runs).  A slab is all-zero between queries: a query over a narrow range zeroes the words
+//     covering [l_q, r_q] when it ends; a query over a wide range instead logs the ranks it evaluates
+//     (a few hundred to a few thousand, next to the slab) and zeroes only their words, so that the
+//     cost of the visited set follows the work of the query, not the width of its range;
 //   * HASH: an open-addressing table in shared memory (no scratch besides the work counter; a
 //     crowded table forgets entries, which costs repeated distance evaluations, never results).
 #include <cstdio>
@@ -65,19 +68,6 @@ __host__ __device__ inline size_t warp_smem_bytes(int pool_slots, int q_len, int
     return (b + 127) & ~(size_t)127;
 }
 inline int query_len(int d) { return (d + 7) / 8 * 8; }
-
-// entry point j of a query range: stateless mixer of (seed, l_q, r_q, j), top 32 bits scaled
-// into [0, w) by a multiply-high (Alg. 2 line 3: uniform sample from [l_q, r_q])
-__device__ __forceinline__ uint32_t entry_point(unsigned long long seed, uint32_t l_q, uint32_t r_q, int j) {
-    unsigned long long x = seed ^ ((unsigned long long)l_q * 0x9E3779B97F4A7C15ull)
-                                ^ ((unsigned long long)r_q * 0xC2B2AE3D27D4EB4Full)
-                                ^ ((unsigned long long)(j + 1) * 0x165667B19E3779F9ull);
-    x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
-    x ^= x >> 27; x *= 0x94D049BB133111EBull;
-    x ^= x >> 31;
-    unsigned long long w = (unsigned long long)(r_q - l_q) + 1ull;
-    return l_q + (uint32_t)(((x >> 32) * w) >> 32);
-}
 
 // test-and-set of rank v in the visited set; true iff v had not been evaluated yet
 template <bool BITMAP>
@@ -160,7 +150,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
         reinterpret_cast<uint32_t*>(S.bar + 2)[1] = 0u;   // copy-timeout flag
     }
     __syncwarp();
-    uint32_t* bitmap = BITMAP ? A.bitmap + (size_t)(blockIdx.x * WARPS_PER_CTA + warp) * A.bitmap_words : nullptr;
+    uint32_t* bitmap = BITMAP ? A.bitmap + (size_t)(blockIdx.x * WARPS_PER_CTA + warp) * A.slab_stride : nullptr;
     const uint32_t lt_mask = (1u << lane) - 1u;
     const uint64_t keep_in_l2 = l2_policy_evict_last();      // for the visited slab of the running query
 
@@ -238,10 +228,16 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                 __syncwarp();
             }
         } else {
+            // Visited slab.  With `slab_clean` it is all-zero here and this query restores that when it
+            // ends: by zeroing the words of its range, or (wide ranges) only the words of the ranks it
+            // logged.  Without it the words of the range are zeroed now.
+            int n_logged = -1;                                      // >= 0: ranks logged so far
             if (BITMAP) {
-                // clear the words that cover [l_q, r_q]
                 const int w0 = l_q >> 5, w1 = r_q >> 5;
-                for (int i = w0 + lane; i <= w1; i += 32) st_u32_l2(bitmap + i, 0u, keep_in_l2);
+                if (!A.slab_clean)
+                    for (int i = w0 + lane; i <= w1; i += 32) st_u32_l2(bitmap + i, 0u, keep_in_l2);
+                else if (A.log_cap > 0 && w1 - w0 >= SPARSE_MIN_WORDS)
+                    n_logged = 0;
             } else {
                 uint4* h4 = reinterpret_cast<uint4*>(S.hash);
                 const uint4 e4 = make_uint4(HASH_EMPTY, HASH_EMPTY, HASH_EMPTY, HASH_EMPTY);
@@ -266,6 +262,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
             }
             FROG_PHASE(0);
             if (COUNT) n_dist += ns;
+            if (BITMAP && n_logged >= 0) n_logged = log_ranks(bitmap + A.bitmap_words, A.log_cap, n_logged, S.cand, ns, lane);
             int first = EVAL(ns, 0u);
             // lines 7-17
             while (first < A.ef_s) {
@@ -401,6 +398,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                         trace_ok = false;
                     }
                 }
+                if (BITMAP && n_logged >= 0) n_logged = log_ranks(bitmap + A.bitmap_words, A.log_cap, n_logged, S.cand, ns, lane);
                 // lines 14-17; a budget above 32 can leave up to 64 survivors: two batches, the pool
                 // after both is the same as after one merge of all of them
                 if (ns > 32) {
@@ -410,16 +408,27 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                     first = EVAL(ns, 0u);
                 }
             }
+            if (BITMAP && A.slab_clean) {
+                // leave the slab all-zero: the words of the logged ranks, or of the whole range
+                if (n_logged >= 0) {
+                    const uint32_t* log = bitmap + A.bitmap_words;
+                    for (int i = lane; i < n_logged; i += 32) st_u32_l2(bitmap + (__ldcg(log + i) >> 5), 0u, keep_in_l2);
+                } else {
+                    const int w0 = l_q >> 5, w1 = r_q >> 5;
+                    for (int i = w0 + lane; i <= w1; i += 32) bitmap[i] = 0u;
+                }
+            }
         }
 
         // ---- line 18: first k of the pool ---------------------------------------------------
         __syncwarp();
+        const bool bad = reinterpret_cast<uint32_t*>(S.bar + 2)[1] != 0u;   // a copy never completed: not valid
         int got = 0;
         for (int j = lane; j < A.k; j += 32) {
             uint64_t key = S.pool[j];
             int32_t oid = -1;
             float dist = __int_as_float(0x7F800000);
-            if (key != KEY_EMPTY) {
+            if (key != KEY_EMPTY && !bad) {
                 oid = __ldg(A.rank2id + key_rank(key));
                 dist = __fsqrt_rn(key_dist2(key));
                 ++got;
@@ -430,7 +439,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
         got = __reduce_add_sync(FULL, got);
         if (got < A.k) st |= FROG_ST_SHORT;
         if (__any_sync(FULL, forgets != 0)) st |= FROG_ST_FORGOT;   // counted per lane
-        if (reinterpret_cast<uint32_t*>(S.bar + 2)[1]) st |= FROG_ST_COPY_TIMEOUT;
+        if (bad) st |= FROG_ST_COPY_TIMEOUT;
         FROG_PHASE(4);
         if (lane == 0) {
             if (A.status) A.status[q] = st;
@@ -487,7 +496,7 @@ frog_order_kernel(const int32_t* __restrict__ lo, const int32_t* __restrict__ hi
     order[pos] = q;
 }
 
-typedef void (*kernel_fn)(const FrogSearchArgs);
+typedef frog_kernel_fn kernel_fn;
 
 template <int MODE, bool BITMAP, bool F16>
 kernel_fn pick_kernel(int ef_s, int* pool_slots) {
@@ -549,6 +558,16 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
         else if (rb == 3072) fn = pick_rowb<3072>(beam_width);
     }
     size_t smem = warp_smem_bytes(pool_slots, query_len(ix->info.d), P.hash_bits, bitmap) * WARPS_PER_CTA;
+    // the trimmed kernel for short fp32 rows (needs the row tensor map); debug_flags bit 2 keeps the generic one
+    if (mode == MODE_FAST && bitmap && !f16 && !P.eager_hash && FROG_GATHER4 && ix->has_tmap_f32 && !(P.debug_flags & 4)) {
+        size_t per_warp = 0;
+        int wpc = 0;
+        kernel_fn lean = froghost::lean_kernel(beam_width, ix->info.d_pad * 4, &per_warp, &wpc);
+        if (lean && wpc == WARPS_PER_CTA) {
+            fn = lean;
+            smem = per_warp * WARPS_PER_CTA;
+        }
+    }
     if (smem > 227 * 1024) return FROG_ERR_UNSUPPORTED;
     FROG_CUDA_TRY(cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
@@ -583,6 +602,12 @@ void set_gather(const frog_index* ix, bool f16, FrogSearchArgs* A) {
 size_t bitmap_words_per_slot(const frog_index* ix) {
     size_t words = ((size_t)ix->info.n + 31) / 32;
     return (words + 31) & ~(size_t)31;
+}
+// entries of the log of evaluated ranks that follows the bits of a slab in the index's own scratch
+// (indexes whose slab never reaches SPARSE_MIN_WORDS have none)
+constexpr int SLAB_LOG_ENTRIES = 8192;
+int slab_log_entries(const frog_index* ix) {
+    return bitmap_words_per_slot(ix) > (size_t)SPARSE_MIN_WORDS ? SLAB_LOG_ENTRIES : 0;
 }
 
 }  // namespace
@@ -695,7 +720,7 @@ int acquire_scratch(frog_index* ix, cudaStream_t s, FrogScratch** out) {
 // Make sure the set owns a visited slab for `slots` resident warps.  Grows (cudaFree + cudaMalloc,
 // after synchronising the device) only when a launch needs more slots than any launch before it.
 int ensure_bitmap(const frog_index* ix, FrogScratch* sc, size_t slots) {
-    const size_t words = bitmap_words_per_slot(ix);
+    const size_t words = bitmap_words_per_slot(ix) + (size_t)slab_log_entries(ix);
     if (sc->d_bitmap && sc->bitmap_slots >= slots) return FROG_OK;
     FROG_CUDA_TRY(cudaDeviceSynchronize());
     if (sc->d_bitmap) FROG_CUDA_TRY(cudaFree(sc->d_bitmap));
@@ -707,6 +732,9 @@ int ensure_bitmap(const frog_index* ix, FrogScratch* sc, size_t slots) {
         set_cuda_error(e);
         return FROG_ERR_NOMEM;
     }
+    // the search kernel keeps every slab all-zero between queries; start it that way
+    FROG_CUDA_TRY(cudaMemset(sc->d_bitmap, 0, slots * words * sizeof(uint32_t)));
+    FROG_CUDA_TRY(cudaDeviceSynchronize());               // before a launch on any (non-blocking) stream
     sc->bitmap_slots = slots;
     return FROG_OK;
 }
@@ -813,6 +841,9 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     A.work_counter = sc->d_work;
     A.bitmap = bitmap ? sc->d_bitmap : nullptr;
     A.bitmap_words = bitmap_words_per_slot(index);
+    A.log_cap = slab_log_entries(index);
+    A.slab_stride = A.bitmap_words + (size_t)A.log_cap;
+    A.slab_clean = 1;
     A.ranges = nullptr;
     A.order = nullptr;
     set_gather(index, P.storage == FROG_STORAGE_F16, &A);
@@ -941,6 +972,9 @@ extern "C" int frog_search_static(const frog_index_t* index, const float* querie
     A.work_counter = scratch;                               // word 0 of the header
     A.bitmap = scratch + STATIC_HEADER_WORDS;
     A.bitmap_words = words;
+    A.slab_stride = words;
+    A.log_cap = 0;
+    A.slab_clean = 0;                                       // the array may hold anything: clear before use
     A.ranges = nullptr;                                     // endpoints and order are computed in the kernel
     A.order = nullptr;
     set_gather(index, P.storage == FROG_STORAGE_F16, &A);

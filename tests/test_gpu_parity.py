@@ -294,6 +294,33 @@ def test_scaled_workloads_match_oracle(libs, cache_dir, name, n, nq):
         gix.close()
 
 
+@pytest.mark.parametrize("name,n,nq", [("sift", 60_000, 300), ("deep1m", 50_000, 300)])
+def test_row_specialised_kernel_at_every_pool_size(libs, cache_dir, name, n, nq):
+    """Rows of 512 and 384 bytes are searched by a kernel specialised for them (every pool size from
+    32 to 512 keys is its own instantiation).  The plain call (which takes it) against the oracle and,
+    inside _gpu_search, against the counting variant of the general kernel, bit for bit; then the
+    general kernel forced by debug_flags bit 2 against the same reference."""
+    from conftest import build_scaled
+    wl, path, ix = build_scaled(libs, cache_dir, name, n, nq)
+    gix = libs.Index.load(path, 0)
+    try:
+        for ef, k, kw in ((24, 10, dict(budget=64)), (64, 64, dict(budget=64, epn=32)), (128, 10, dict(budget=64)),
+                          (200, 100, dict(budget=48)), (256, 10, dict(budget=64, max_iters=40)),
+                          (512, 10, dict(budget=64)), (96, 10, dict(budget=64, exact_below=2000)),
+                          (40, 10, dict(budget=64, no_hotspot=1, seed=9))):
+            ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef, epn=kw.get("epn", 16), B=kw["budget"],
+                                max_iters=kw.get("max_iters", 0), exact_below=kw.get("exact_below", 0),
+                                no_hotspot=bool(kw.get("no_hotspot", 0)), seed=kw.get("seed", 0))
+            got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, k, ef, **kw)
+            _assert_parity(got, ref)
+            q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
+            ids, dists = gix.search(q, lo, hi, k, ef, params=libs.Params(debug_flags=4, **kw))
+            torch.cuda.synchronize()
+            assert np.array_equal(ids.cpu().numpy(), ref.ids) and np.array_equal(dists.cpu().numpy(), ref.dists)
+    finally:
+        gix.close()
+
+
 def test_odd_dimension(libs, cache_dir):
     rng = np.random.default_rng(2)
     V = rng.standard_normal((3000, 10)).astype(np.float32)

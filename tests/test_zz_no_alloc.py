@@ -1,10 +1,12 @@
 """frog_search_static: the search entry point for callers that may not allocate device memory
 (stream capture, fixed memory budgets, a foreign caching allocator owning the free memory).
 
-Its scratch is a fixed device array inside the library instead of buffers owned by the index, so
-the check is simply that it returns what the regular entry point returns -- twice in a row, since
-the array keeps the previous call's contents and a stale counter or stale visited bits would show
-up on the second call.  Collected last so that a failure here cannot hide other results."""
+Its scratch is a fixed device array inside the library instead of buffers owned by the index.  The
+check: it returns what the CPU oracle computes for the same index (and therefore what the regular
+entry point returns) -- twice in a row, since the array keeps the previous call's contents and a stale
+counter or stale visited bits would show up on the second call -- and the device's free-memory reading
+is the same before and after a call once the first call has done its one-time set-up.  Collected last
+so that a failure here cannot hide other results."""
 import numpy as np
 import pytest
 
@@ -18,31 +20,41 @@ def _run(libs, n, nq, beam, budget):
     import tempfile
 
     import datagen
+    import oracle
 
     wl = datagen.make_workload("sift", n=n, nq=nq)
     with tempfile.TemporaryDirectory() as tmp:
         path = os.path.join(tmp, "static.idx")
         libs.build_index(wl.vectors, wl.attrs, path, seed=wl.seed)
         ix = libs.Index.load(path, 0)
+        ref = oracle.search(oracle.load_index(path), wl.queries, wl.lo, wl.hi, wl.k, beam, B=budget)
     q = torch.from_numpy(wl.queries).cuda()
     lo = torch.from_numpy(wl.lo).cuda()
     hi = torch.from_numpy(wl.hi).cuda()
     prm = libs.Params(budget=budget)
-    ref_ids, ref_d = ix.search(q, lo, hi, wl.k, beam, params=prm)
+    # the regular entry point agrees with the oracle too (it allocates its scratch on first use)
+    reg_ids, reg_d = ix.search(q, lo, hi, wl.k, beam, params=prm)
     torch.cuda.synchronize()
-    ref_ids, ref_d = ref_ids.cpu().numpy(), ref_d.cpu().numpy()
+    assert np.array_equal(reg_ids.cpu().numpy(), ref.ids)
     out_ids = torch.empty((nq, wl.k), dtype=torch.int32, device="cuda")
     out_d = torch.empty((nq, wl.k), dtype=torch.float32, device="cuda")
-    for call in range(2):
+    fin = np.isfinite(ref.dists)
+    for call in range(3):
         out_ids.fill_(-7)
         out_d.fill_(-7.0)
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
         ix.search_static(q, lo, hi, wl.k, beam, out_ids=out_ids, out_dists=out_d, params=prm)
         torch.cuda.synchronize()
-        assert np.array_equal(out_ids.cpu().numpy(), ref_ids), f"ids differ on call {call}"
-        fin = np.isfinite(ref_d)
+        free_after, _ = torch.cuda.mem_get_info()
+        if call > 0:
+            # nothing was allocated (or freed) on the device by the call; the first call on a device may
+            # load the library's module and is not held to this
+            assert free_after == free_before, f"free device memory changed across call {call}"
+        assert np.array_equal(out_ids.cpu().numpy(), ref.ids), f"ids differ from the oracle on call {call}"
         got = out_d.cpu().numpy()
         assert np.array_equal(np.isfinite(got), fin)
-        assert np.allclose(got[fin], ref_d[fin], rtol=1e-4, atol=0), f"distances differ on call {call}"
+        assert np.allclose(got[fin], ref.dists[fin], rtol=1e-4, atol=0), f"distances differ on call {call}"
     return ix
 
 
