@@ -263,6 +263,10 @@ __device__ __forceinline__ void tma_load_1d_l2(void* dst_smem, const void* src_g
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                  ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)), "l"(l2_policy) : "memory");
 }
+// credit `bytes` to the barrier's pending transaction count without a copy (a row slot left empty)
+__device__ __forceinline__ void mbar_complete_tx_dummy(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
 // Wait for the phase of parity `phase`; bounded: gives up after 2^22 polls and reports false (the
 // caller flags the query instead of hanging the GPU).  try_wait already parks the thread for a
 // hardware-chosen interval per poll; passing an explicit suspend-time hint measured 7 % slower.
@@ -609,6 +613,70 @@ __device__ __forceinline__ uint32_t merge_batch(uint64_t* pool, uint64_t my_key,
     }
     __syncwarp();
     return first_pos(m1);
+}
+
+// The same merge for large pools without holding the pool in registers (EPL >= 8 would cost 16+
+// registers per lane and with them a quarter of the resident warps).  Keys must be unique (exact
+// visited set).  A new key's final position is (#pool keys below it, by binary search in shared
+// memory) + (#new keys below it, by shuffles).  A pool key at position i moves up by the number of
+// new keys that land at or below i -- a non-decreasing step function of i, so the entries that do
+// not move form a prefix and the rest can be shifted IN PLACE chunk by chunk from the top: the 32
+// keys of a chunk are read, then written to i + shift (into their own chunk or the one above, whose
+// old contents have already moved on).  Then the new keys drop into the slots left free.  Returns
+// the position of the first entry whose flag is 0 (0xFFFF = none).
+template <int EPL>
+__device__ __forceinline__ uint32_t merge_inplace(uint64_t* pool, uint64_t my_key, int ef_s, int lane) {
+    constexpr int POOL = 32 * EPL;
+    const uint64_t worst = pool[ef_s - 1];
+    if ((my_key | 1ull) >= (worst | 1ull)) my_key = KEY_EMPTY;      // a full pool rejects what is not better
+    const uint32_t have = __ballot_sync(FULL, my_key != KEY_EMPTY);
+    if (have) {
+        const uint64_t mk = my_key | 1ull;
+        int pp = POOL;                                              // pool keys below mine (POOL: none of mine)
+        if (my_key != KEY_EMPTY) {
+            int lo = 0, hi = POOL;
+#pragma unroll 1
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if ((pool[mid] | 1ull) < mk) lo = mid + 1; else hi = mid;
+            }
+            pp = lo;
+        }
+        int rnew = 0;                                               // new keys below mine
+        const uint32_t my_lo = (uint32_t)mk, my_hi = (uint32_t)(mk >> 32);
+#pragma unroll 1
+        for (uint32_t msk = have; msk; msk &= msk - 1) {
+            const int j = __ffs(msk) - 1;
+            const uint64_t x = ((uint64_t)__shfl_sync(FULL, my_hi, j) << 32) | __shfl_sync(FULL, my_lo, j);
+            rnew += (x < mk) ? 1 : 0;
+        }
+        const int min_pp = (int)__reduce_min_sync(FULL, (unsigned)pp);
+#pragma unroll 1
+        for (int e = EPL - 1; e >= 0 && 32 * e + 31 >= min_pp; --e) {
+            const int i = 32 * e + lane;
+            const uint64_t key = pool[i];
+            int shift = 0;
+#pragma unroll 1
+            for (uint32_t msk = have; msk; msk &= msk - 1) {
+                const int ppj = __shfl_sync(FULL, pp, __ffs(msk) - 1);
+                shift += (ppj <= i) ? 1 : 0;
+            }
+            __syncwarp();                                           // every lane holds its key of this chunk
+            if (key != KEY_EMPTY && shift > 0 && i + shift < ef_s) pool[i + shift] = key;
+            __syncwarp();
+        }
+        if (my_key != KEY_EMPTY && pp + rnew < ef_s) pool[pp + rnew] = my_key;
+        __syncwarp();
+    }
+#pragma unroll 1
+    for (int e = 0; e < EPL; ++e) {
+        const int i = 32 * e + lane;
+        const uint64_t key = pool[i];
+        const uint32_t un = __ballot_sync(FULL, key != KEY_EMPTY && !(key & 1ull) && i < ef_s);
+        if (un) return (uint32_t)(32 * e + __ffs(un) - 1);
+        if (__any_sync(FULL, key == KEY_EMPTY)) break;              // the tail is empty from here on
+    }
+    return 0xFFFFu;
 }
 
 // smallest key of the warp under the order key | 1 (KEY_EMPTY if no lane has one)

@@ -25,7 +25,10 @@ namespace {
 
 constexpr int LEAN_WARPS = 2;      // warps per CTA; they never synchronise with each other
 #ifndef FROG_LEAN_NSLOT_384
-#define FROG_LEAN_NSLOT_384 3      // quads (4 rows each) in the stage ring for 384-byte rows
+#define FROG_LEAN_NSLOT_384 2      // quads (4 rows each) in the stage ring for 384-byte rows
+#endif
+#ifndef FROG_LEAN_MINB
+#define FROG_LEAN_MINB 16          // resident CTAs per SM the register allocation aims at (pools up to 128 keys)
 #endif
 #ifndef FROG_LEAN_NSLOT_512
 #define FROG_LEAN_NSLOT_512 2      // ... for 512-byte rows
@@ -87,6 +90,25 @@ __device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanS
     if (lane < 3) S.cand[ns + lane] = (uint32_t)A.n + 1u + (uint32_t)lane;    // rows beyond the tensor: zeros
     __syncwarp();
     const uint64_t policy = l2_policy_evict_first();                           // rows are read about once per batch
+#ifdef FROG_LEAN_BULK1D
+    // one plain bulk copy per row, issued by lanes 0..3 of the quad (experiment: no tensor map)
+    auto issue = [&](int g, int slot) {
+        uint64_t* b = S.bar + slot;
+        if (lane == 0) mbar_expect_tx(b, (uint32_t)L::QUAD);
+        __syncwarp();
+        if (lane < 4) {
+            const uint32_t r = S.cand[4 * g + lane];
+            if (r < (uint32_t)A.n)
+                tma_load_1d_l2(S.stage + slot * L::QUAD + lane * ROWB, reinterpret_cast<const char*>(A.rows) + (size_t)r * ROWB,
+                               (uint32_t)ROWB, b, policy);
+            else
+                mbar_complete_tx_dummy(b, (uint32_t)ROWB);
+        }
+    };
+#pragma unroll
+    for (int g = 0; g < L::NSLOT; ++g)
+        if (g < groups) issue(g, g);
+#else
     auto issue = [&](int g, int slot) {
         uint64_t* b = S.bar + slot;
         mbar_expect_tx(b, (uint32_t)L::QUAD);
@@ -98,6 +120,7 @@ __device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanS
         for (int g = 0; g < L::NSLOT; ++g)
             if (g < groups) issue(g, g);
     }
+#endif
     const int team = lane >> 3, sub = lane & 7;
     const char* mine = S.stage + team * ROWB + sub * 16;
     int slot = 0;
@@ -122,7 +145,11 @@ __device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanS
         a = a + __shfl_xor_sync(FULL, a, 1);
         if (sub == 0) S.d2[4 * g + team] = a;
         __syncwarp();                                       // every lane is done reading this quad
+#ifdef FROG_LEAN_BULK1D
+        if (g + L::NSLOT < groups) issue(g + L::NSLOT, slot);
+#else
         if (lane == 0 && g + L::NSLOT < groups) issue(g + L::NSLOT, slot);
+#endif
         slot = (slot + 1 == L::NSLOT) ? 0 : slot + 1;
     }
     __syncwarp();
@@ -133,6 +160,9 @@ template <int EPL, int ROWB>
 __device__ __forceinline__ int lean_merge(const LeanSmem<EPL, ROWB>& S, int ns, int ef_s, uint32_t new_flag, int off, int lane) {
     const int j = off + lane;
     const uint64_t key = (j < ns) ? make_key(S.d2[j], S.cand[j], new_flag) : KEY_EMPTY;
+#ifndef FROG_LEAN_REGISTER_MERGE
+    if (EPL >= 8) return (int)merge_inplace<EPL>(S.pool, key, ef_s, lane);      // pools of 256 and 512 keys
+#endif
     return (int)merge_batch<EPL, true>(S.pool, key, ef_s, lane);
 }
 
@@ -155,7 +185,11 @@ __device__ __noinline__ int lean_merge_cold(unsigned char* base, int ns, int ef_
 }
 
 template <int EPL, int ROWB>
-__global__ void __launch_bounds__(LEAN_WARPS * 32, EPL <= 4 ? 16 : EPL == 8 ? 12 : 10)
+#ifdef FROG_LEAN_REGISTER_MERGE
+__global__ void __launch_bounds__(LEAN_WARPS * 32, EPL <= 4 ? FROG_LEAN_MINB : EPL == 8 ? 12 : 10)
+#else
+__global__ void __launch_bounds__(LEAN_WARPS * 32, FROG_LEAN_MINB)
+#endif
 frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
     using L = Lean<EPL, ROWB>;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -176,7 +210,13 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
 #endif
     uint32_t* bitmap = A.bitmap + (size_t)(blockIdx.x * LEAN_WARPS + warp) * A.slab_stride;
     const uint32_t lt_mask = (1u << lane) - 1u;
+#if defined(FROG_LEAN_SLAB_POLICY) && FROG_LEAN_SLAB_POLICY == 1
+    const uint64_t keep_in_l2 = l2_policy_evict_normal();
+#elif defined(FROG_LEAN_SLAB_POLICY) && FROG_LEAN_SLAB_POLICY == 2
+    const uint64_t keep_in_l2 = l2_policy_evict_first();
+#else
     const uint64_t keep_in_l2 = l2_policy_evict_last();      // for the visited slab of the running query
+#endif
 
     for (;;) {
         int q = 0;
