@@ -72,7 +72,9 @@ typedef struct {
     int32_t debug_flags;/* bit 0: with `trace`, record per-phase cycle counts instead of EN lists;
                            bit 1: process queries in input order (no heaviest-first planning pass);
                            bit 2: use the general kernel where a kernel specialised for the row size exists
-                                  (same results; for comparing the two) */
+                                  (same results; for comparing the two);
+                           bit 3: use the visited hash table (see FROG_VISITED_AUTO) on small indexes too;
+                           bits 8-11: log2 of that table's slots, 6..12 (0 = 12), to make queries outgrow it */
     int32_t exact_below;/* ranges holding at most max(beam_width, exact_below) objects are answered by
                            scanning their contiguous rank slab (exact, status FROG_ST_EXACT) instead of
                            the graph search; 0 = default: only ranges that fit the pool.  Not in the
@@ -92,7 +94,11 @@ typedef struct {
 /* Visited set (hashCheck of Alg. 2).  BITMAP: one bit per rank in a per-warp slab of device
  * scratch memory owned by the index (n/8 bytes per resident warp, allocated on first use, exact).
  * HASH: a bounded table in shared memory, no scratch; a crowded table drops entries, which repeats
- * distance evaluations but never changes results.  AUTO = BITMAP, HASH if the slabs do not fit. */
+ * distance evaluations but never changes results.  AUTO = BITMAP (HASH if the slabs do not fit);
+ * for indexes of 4,194,304 objects and more searched with 384- or 512-byte rows and beam_width <= 64, AUTO
+ * keeps the set in a 16 KB hash table of ranks per resident warp instead (exact; small enough to stay
+ * in L2, where the bitmap of a large index costs a DRAM read-modify-write per candidate); a query
+ * that fills half the table moves to its bitmap slab.  The results do not depend on the form. */
 #define FROG_VISITED_AUTO 0
 #define FROG_VISITED_BITMAP 1
 #define FROG_VISITED_HASH 2

@@ -263,10 +263,6 @@ __device__ __forceinline__ void tma_load_1d_l2(void* dst_smem, const void* src_g
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                  ::"r"(smem_u32(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)), "l"(l2_policy) : "memory");
 }
-// credit `bytes` to the barrier's pending transaction count without a copy (a row slot left empty)
-__device__ __forceinline__ void mbar_complete_tx_dummy(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
 // Wait for the phase of parity `phase`; bounded: gives up after 2^22 polls and reports false (the
 // caller flags the query instead of hanging the GPU).  try_wait already parks the thread for a
 // hardware-chosen interval per poll; passing an explicit suspend-time hint measured 7 % slower.
@@ -615,70 +611,6 @@ __device__ __forceinline__ uint32_t merge_batch(uint64_t* pool, uint64_t my_key,
     return first_pos(m1);
 }
 
-// The same merge for large pools without holding the pool in registers (EPL >= 8 would cost 16+
-// registers per lane and with them a quarter of the resident warps).  Keys must be unique (exact
-// visited set).  A new key's final position is (#pool keys below it, by binary search in shared
-// memory) + (#new keys below it, by shuffles).  A pool key at position i moves up by the number of
-// new keys that land at or below i -- a non-decreasing step function of i, so the entries that do
-// not move form a prefix and the rest can be shifted IN PLACE chunk by chunk from the top: the 32
-// keys of a chunk are read, then written to i + shift (into their own chunk or the one above, whose
-// old contents have already moved on).  Then the new keys drop into the slots left free.  Returns
-// the position of the first entry whose flag is 0 (0xFFFF = none).
-template <int EPL>
-__device__ __forceinline__ uint32_t merge_inplace(uint64_t* pool, uint64_t my_key, int ef_s, int lane) {
-    constexpr int POOL = 32 * EPL;
-    const uint64_t worst = pool[ef_s - 1];
-    if ((my_key | 1ull) >= (worst | 1ull)) my_key = KEY_EMPTY;      // a full pool rejects what is not better
-    const uint32_t have = __ballot_sync(FULL, my_key != KEY_EMPTY);
-    if (have) {
-        const uint64_t mk = my_key | 1ull;
-        int pp = POOL;                                              // pool keys below mine (POOL: none of mine)
-        if (my_key != KEY_EMPTY) {
-            int lo = 0, hi = POOL;
-#pragma unroll 1
-            while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
-                if ((pool[mid] | 1ull) < mk) lo = mid + 1; else hi = mid;
-            }
-            pp = lo;
-        }
-        int rnew = 0;                                               // new keys below mine
-        const uint32_t my_lo = (uint32_t)mk, my_hi = (uint32_t)(mk >> 32);
-#pragma unroll 1
-        for (uint32_t msk = have; msk; msk &= msk - 1) {
-            const int j = __ffs(msk) - 1;
-            const uint64_t x = ((uint64_t)__shfl_sync(FULL, my_hi, j) << 32) | __shfl_sync(FULL, my_lo, j);
-            rnew += (x < mk) ? 1 : 0;
-        }
-        const int min_pp = (int)__reduce_min_sync(FULL, (unsigned)pp);
-#pragma unroll 1
-        for (int e = EPL - 1; e >= 0 && 32 * e + 31 >= min_pp; --e) {
-            const int i = 32 * e + lane;
-            const uint64_t key = pool[i];
-            int shift = 0;
-#pragma unroll 1
-            for (uint32_t msk = have; msk; msk &= msk - 1) {
-                const int ppj = __shfl_sync(FULL, pp, __ffs(msk) - 1);
-                shift += (ppj <= i) ? 1 : 0;
-            }
-            __syncwarp();                                           // every lane holds its key of this chunk
-            if (key != KEY_EMPTY && shift > 0 && i + shift < ef_s) pool[i + shift] = key;
-            __syncwarp();
-        }
-        if (my_key != KEY_EMPTY && pp + rnew < ef_s) pool[pp + rnew] = my_key;
-        __syncwarp();
-    }
-#pragma unroll 1
-    for (int e = 0; e < EPL; ++e) {
-        const int i = 32 * e + lane;
-        const uint64_t key = pool[i];
-        const uint32_t un = __ballot_sync(FULL, key != KEY_EMPTY && !(key & 1ull) && i < ef_s);
-        if (un) return (uint32_t)(32 * e + __ffs(un) - 1);
-        if (__any_sync(FULL, key == KEY_EMPTY)) break;              // the tail is empty from here on
-    }
-    return 0xFFFFu;
-}
-
 // smallest key of the warp under the order key | 1 (KEY_EMPTY if no lane has one)
 __device__ __forceinline__ uint64_t warp_min_key(uint64_t key) {
     const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key | 1u;
@@ -712,6 +644,62 @@ __device__ __forceinline__ int log_ranks(uint32_t* log, int cap, int n_logged, c
     if (lane < ns) __stcg(log + n_logged + lane, cand[lane]);
     if (lane + 32 < ns) __stcg(log + n_logged + lane + 32, cand[lane + 32]);
     return n_logged + ns;
+}
+
+// ---- visited TABLE: an exact hash set in global memory, small enough to stay in L2 ---------------
+// 4-slot buckets of ranks (16 bytes), 0xFFFFFFFF = empty, linear probing over buckets.  A key is
+// looked up with one 16-byte load of its bucket and, if absent, claimed with a compare-and-swap on
+// the first empty slot; losing the slot to another key means looking at the bucket again.  Slots
+// never become empty while a query runs, so a key absent from a bucket with a free slot is absent
+// from the table.  The caller keeps the table at most half full.
+constexpr uint32_t TABLE_EMPTY = 0xFFFFFFFFu;
+__device__ __forceinline__ uint4 ld_bucket_l2(const uint32_t* p, uint64_t policy) {
+    uint4 v;
+    asm volatile("ld.global.cg.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(policy) : "memory");
+    return v;
+}
+// (the compare-and-swap form of atom takes no L2 cache hint; the bucket loads carry it)
+__device__ __forceinline__ uint32_t atomic_cas_l2(uint32_t* p, uint32_t cmp, uint32_t val, uint64_t) {
+    return atomicCAS(p, cmp, val);
+}
+__device__ __forceinline__ uint32_t table_bucket(uint32_t v, int table_bits) {
+    return (v * 0x9E3779B1u) >> (34 - table_bits);           // table_bits - 2 bucket bits
+}
+// slot of the bucket that holds v (-1), the first empty slot (0..3), or 4 when the bucket is full of other keys
+__device__ __forceinline__ int bucket_find(const uint4& b, uint32_t v) {
+    if (b.x == v || b.y == v || b.z == v || b.w == v) return -1;
+    return b.x == TABLE_EMPTY ? 0 : b.y == TABLE_EMPTY ? 1 : b.z == TABLE_EMPTY ? 2 : b.w == TABLE_EMPTY ? 3 : 4;
+}
+// Test-and-insert of up to two keys per lane (a lane's probes of both keys are in flight together).
+// fa / fb: the key was not in the table and is now.  Returns false if a probe sequence ran into its limit.
+__device__ __forceinline__ bool table_insert2(uint32_t* table, int table_bits, uint32_t va, bool ha, uint32_t vb, bool hb,
+                                              bool& fa, bool& fb, uint64_t policy) {
+    const uint32_t bmask = (1u << (table_bits - 2)) - 1u;
+    uint32_t ka = table_bucket(va, table_bits), kb = table_bucket(vb, table_bits);
+    bool pa = ha, pb = hb;
+    fa = fb = false;
+#pragma unroll 1
+    for (int it = 0; it < 4096 && __any_sync(FULL, pa || pb); ++it) {
+        uint4 ba = make_uint4(0, 0, 0, 0), bb = make_uint4(0, 0, 0, 0);
+        if (pa) ba = ld_bucket_l2(table + 4 * ka, policy);
+        if (pb) bb = ld_bucket_l2(table + 4 * kb, policy);
+        const int ja = pa ? bucket_find(ba, va) : -1, jb = pb ? bucket_find(bb, vb) : -1;
+        uint32_t oa = va, ob = vb;
+        if (pa && ja >= 0 && ja < 4) oa = atomic_cas_l2(table + 4 * ka + ja, TABLE_EMPTY, va, policy);
+        if (pb && jb >= 0 && jb < 4) ob = atomic_cas_l2(table + 4 * kb + jb, TABLE_EMPTY, vb, policy);
+        if (pa) {
+            if (ja == 4) ka = (ka + 1) & bmask;
+            else if (ja < 0 || oa == va) pa = false;                // found, or another lane put it there just now
+            else if (oa == TABLE_EMPTY) { fa = true; pa = false; }
+        }
+        if (pb) {
+            if (jb == 4) kb = (kb + 1) & bmask;
+            else if (jb < 0 || ob == vb) pb = false;
+            else if (ob == TABLE_EMPTY) { fb = true; pb = false; }
+        }
+    }
+    return !__any_sync(FULL, pa || pb);
 }
 
 }  // namespace frogdev

@@ -115,6 +115,7 @@ extern "C" void frog_index_free(frog_index_t* ix) {
         for (int i = 0; i < ix->n_scratch; ++i) {
             cudaFree(ix->scratch[i].d_work);
             cudaFree(ix->scratch[i].d_bitmap);
+            cudaFree(ix->scratch[i].d_table);
             cudaFree(ix->scratch[i].d_plan);
             if (ix->scratch[i].done) cudaEventDestroy(ix->scratch[i].done);
         }

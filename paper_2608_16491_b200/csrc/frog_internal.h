@@ -15,6 +15,8 @@ struct FrogScratch {
     unsigned int* d_work = nullptr;  // 1 KB
     uint32_t* d_bitmap = nullptr;    // bitmap_slots x (words of visited bits + log of evaluated ranks)
     size_t bitmap_slots = 0;
+    uint32_t* d_table = nullptr;     // table_slots visited hash tables of FROG_TABLE_SLOTS ranks (all 0xFFFFFFFF at rest)
+    size_t table_slots = 0;
     int32_t* d_plan = nullptr;       // per query: rank interval (2 ints) and processing order (1 int)
     size_t plan_queries = 0;
     cudaEvent_t done = nullptr;
@@ -22,6 +24,7 @@ struct FrogScratch {
     unsigned long long tick = 0;
 };
 constexpr int FROG_SCRATCH_SETS = 4;
+constexpr int FROG_TABLE_BITS = 12;    // 4,096 ranks = 16 KB per resident warp: 78 MB for a full grid, inside L2
 
 struct frog_index {
     frog_index_info_t info;
@@ -74,6 +77,9 @@ struct FrogSearchArgs {
     int log_cap;               // entries of the per-warp log of evaluated ranks that follows the bits (0: none)
     int slab_clean;            // nonzero: every slab is all-zero between queries (the kernel restores that
                                // when a query ends); zero: a query clears the words of its range before use
+    uint32_t* table;           // visited hash tables (1 << table_bits ranks per resident warp, all empty
+                               // between queries), or null
+    int table_bits;
     const int2* ranges;        // precomputed [l_q, r_q] per query, or null: computed in the kernel
     const int32_t* order;      // processing order (heaviest first), or null: input order
     const void* rows;          // gather source: fp32 vectors, or their fp16 copy
@@ -88,12 +94,13 @@ typedef void (*frog_kernel_fn)(const FrogSearchArgs);
 
 namespace froghost {
 // frog_search_lean.cu: the trimmed kernel for 384- and 512-byte fp32 rows (null: shape not covered)
-frog_kernel_fn lean_kernel(int ef_s, int row_bytes, size_t* smem_per_warp, int* warps_per_cta);
+frog_kernel_fn lean_kernel(int ef_s, int row_bytes, bool table, size_t* smem_per_warp, int* warps_per_cta);
 void set_cuda_error(cudaError_t e);
 int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in, frog_params_t* out);
 bool make_row_tensor_map(const void* base, bool f16, int row_elems, size_t row_bytes, size_t n, CUtensorMap* out);
 int acquire_scratch(frog_index* ix, cudaStream_t s, FrogScratch** out);
 int ensure_bitmap(const frog_index* ix, FrogScratch* sc, size_t slots);
+int ensure_table(FrogScratch* sc, size_t slots);
 int ensure_plan(FrogScratch* sc, size_t nq);
 }  // namespace froghost
 

@@ -517,14 +517,18 @@ kernel_fn pick_rowb(int ef_s) {
     return frog_search_kernel<16, MODE, true, false, ROWB>;
 }
 
+size_t bitmap_words_per_slot(const frog_index* ix);
+constexpr int TABLE_MIN_SLAB_WORDS = 1 << 17;     // 512 KB of visited bits per warp
+
 struct LaunchPlan {
     kernel_fn fn;
     int grid, block, ctas_per_sm;
     size_t smem;
+    bool table;        // the kernel keeps its visited sets in the L2-resident hash tables
 };
 
 int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, int mode, bool bitmap, int nq,
-                LaunchPlan* out) {
+                LaunchPlan* out, bool allow_table = true) {
     int pool_slots = 0;
     kernel_fn fn;
     const bool f16 = P.storage == FROG_STORAGE_F16;
@@ -558,14 +562,27 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
         else if (rb == 3072) fn = pick_rowb<3072>(beam_width);
     }
     size_t smem = warp_smem_bytes(pool_slots, query_len(ix->info.d), P.hash_bits, bitmap) * WARPS_PER_CTA;
+    bool table = false;
     // the trimmed kernel for short fp32 rows (needs the row tensor map); debug_flags bit 2 keeps the generic one
     if (mode == MODE_FAST && bitmap && !f16 && !P.eager_hash && FROG_GATHER4 && ix->has_tmap_f32 && !(P.debug_flags & 4)) {
         size_t per_warp = 0;
         int wpc = 0;
-        kernel_fn lean = froghost::lean_kernel(beam_width, ix->info.d_pad * 4, &per_warp, &wpc);
+        // visited hash table instead of the bitmap: where the slabs are far too large for L2 (indexes of
+        // 4,194,304 objects and more: measured 1.26x faster at 10M objects, 0.85x at 1M, where the bits a
+        // query touches still fit L2) and the pool is small enough for a query to fit the table as a rule;
+        // FROG_VISITED_BITMAP keeps the bitmap
+        table = allow_table && P.visited == FROG_VISITED_AUTO && beam_width <= 64 &&
+                (bitmap_words_per_slot(ix) >= (size_t)TABLE_MIN_SLAB_WORDS || (P.debug_flags & 8));
+        kernel_fn lean = froghost::lean_kernel(beam_width, ix->info.d_pad * 4, table, &per_warp, &wpc);
+        if (!lean && table) {
+            table = false;
+            lean = froghost::lean_kernel(beam_width, ix->info.d_pad * 4, false, &per_warp, &wpc);
+        }
         if (lean && wpc == WARPS_PER_CTA) {
             fn = lean;
             smem = per_warp * WARPS_PER_CTA;
+        } else {
+            table = false;
         }
     }
     if (smem > 227 * 1024) return FROG_ERR_UNSUPPORTED;
@@ -583,6 +600,7 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
     out->block = WARPS_PER_CTA * 32;
     out->ctas_per_sm = per_sm;
     out->smem = smem;
+    out->table = table;
     return FROG_OK;
 }
 
@@ -739,6 +757,26 @@ int ensure_bitmap(const frog_index* ix, FrogScratch* sc, size_t slots) {
     return FROG_OK;
 }
 
+// Visited hash tables for `slots` resident warps, all entries empty (the kernel leaves them so).
+int ensure_table(FrogScratch* sc, size_t slots) {
+    if (sc->d_table && sc->table_slots >= slots) return FROG_OK;
+    FROG_CUDA_TRY(cudaDeviceSynchronize());
+    if (sc->d_table) FROG_CUDA_TRY(cudaFree(sc->d_table));
+    sc->d_table = nullptr;
+    sc->table_slots = 0;
+    const size_t bytes = (slots << FROG_TABLE_BITS) * sizeof(uint32_t);
+    cudaError_t e = cudaMalloc(&sc->d_table, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        set_cuda_error(e);
+        return FROG_ERR_NOMEM;
+    }
+    FROG_CUDA_TRY(cudaMemset(sc->d_table, 0xFF, bytes));
+    FROG_CUDA_TRY(cudaDeviceSynchronize());
+    sc->table_slots = slots;
+    return FROG_OK;
+}
+
 // Per-query planning scratch: 3 ints per query, grown when a batch is larger than any before.
 int ensure_plan(FrogScratch* sc, size_t nq) {
     if (sc->d_plan && sc->plan_queries >= nq) return FROG_OK;
@@ -808,6 +846,10 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
         }
         if (rc) return rc;
     }
+    if (plan.table && froghost::ensure_table(sc, (size_t)plan.grid * WARPS_PER_CTA) != FROG_OK) {
+        rc = plan_launch(index, beam_width, P, mode, bitmap, nq, &plan, false);     // no room: bitmap only
+        if (rc) return rc;
+    }
 
     FrogSearchArgs A;
     A.sorted_attr = index->d_sorted_attr;
@@ -844,6 +886,10 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     A.log_cap = slab_log_entries(index);
     A.slab_stride = A.bitmap_words + (size_t)A.log_cap;
     A.slab_clean = 1;
+    A.table = plan.table ? sc->d_table : nullptr;
+    A.table_bits = FROG_TABLE_BITS;
+    if (((P.debug_flags >> 8) & 15) >= 6 && ((P.debug_flags >> 8) & 15) <= FROG_TABLE_BITS)
+        A.table_bits = (P.debug_flags >> 8) & 15;           // tests: a small table, so that queries outgrow it
     A.ranges = nullptr;
     A.order = nullptr;
     set_gather(index, P.storage == FROG_STORAGE_F16, &A);
@@ -935,7 +981,7 @@ extern "C" int frog_search_static(const frog_index_t* index, const float* querie
     rc = static_scratch_for_device(index->info.device, &scratch);
     if (rc) return rc;
     LaunchPlan plan;
-    rc = plan_launch(index, beam_width, P, MODE_FAST, true, nq, &plan);
+    rc = plan_launch(index, beam_width, P, MODE_FAST, true, nq, &plan, false);
     if (rc) return rc;
     const int max_ctas = (int)(fit / WARPS_PER_CTA);
     if (plan.grid > max_ctas) plan.grid = max_ctas;
@@ -975,6 +1021,8 @@ extern "C" int frog_search_static(const frog_index_t* index, const float* querie
     A.slab_stride = words;
     A.log_cap = 0;
     A.slab_clean = 0;                                       // the array may hold anything: clear before use
+    A.table = nullptr;
+    A.table_bits = 0;
     A.ranges = nullptr;                                     // endpoints and order are computed in the kernel
     A.order = nullptr;
     set_gather(index, P.storage == FROG_STORAGE_F16, &A);

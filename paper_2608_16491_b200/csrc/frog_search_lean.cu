@@ -90,25 +90,6 @@ __device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanS
     if (lane < 3) S.cand[ns + lane] = (uint32_t)A.n + 1u + (uint32_t)lane;    // rows beyond the tensor: zeros
     __syncwarp();
     const uint64_t policy = l2_policy_evict_first();                           // rows are read about once per batch
-#ifdef FROG_LEAN_BULK1D
-    // one plain bulk copy per row, issued by lanes 0..3 of the quad (experiment: no tensor map)
-    auto issue = [&](int g, int slot) {
-        uint64_t* b = S.bar + slot;
-        if (lane == 0) mbar_expect_tx(b, (uint32_t)L::QUAD);
-        __syncwarp();
-        if (lane < 4) {
-            const uint32_t r = S.cand[4 * g + lane];
-            if (r < (uint32_t)A.n)
-                tma_load_1d_l2(S.stage + slot * L::QUAD + lane * ROWB, reinterpret_cast<const char*>(A.rows) + (size_t)r * ROWB,
-                               (uint32_t)ROWB, b, policy);
-            else
-                mbar_complete_tx_dummy(b, (uint32_t)ROWB);
-        }
-    };
-#pragma unroll
-    for (int g = 0; g < L::NSLOT; ++g)
-        if (g < groups) issue(g, g);
-#else
     auto issue = [&](int g, int slot) {
         uint64_t* b = S.bar + slot;
         mbar_expect_tx(b, (uint32_t)L::QUAD);
@@ -120,7 +101,6 @@ __device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanS
         for (int g = 0; g < L::NSLOT; ++g)
             if (g < groups) issue(g, g);
     }
-#endif
     const int team = lane >> 3, sub = lane & 7;
     const char* mine = S.stage + team * ROWB + sub * 16;
     int slot = 0;
@@ -145,11 +125,7 @@ __device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanS
         a = a + __shfl_xor_sync(FULL, a, 1);
         if (sub == 0) S.d2[4 * g + team] = a;
         __syncwarp();                                       // every lane is done reading this quad
-#ifdef FROG_LEAN_BULK1D
-        if (g + L::NSLOT < groups) issue(g + L::NSLOT, slot);
-#else
         if (lane == 0 && g + L::NSLOT < groups) issue(g + L::NSLOT, slot);
-#endif
         slot = (slot + 1 == L::NSLOT) ? 0 : slot + 1;
     }
     __syncwarp();
@@ -160,9 +136,6 @@ template <int EPL, int ROWB>
 __device__ __forceinline__ int lean_merge(const LeanSmem<EPL, ROWB>& S, int ns, int ef_s, uint32_t new_flag, int off, int lane) {
     const int j = off + lane;
     const uint64_t key = (j < ns) ? make_key(S.d2[j], S.cand[j], new_flag) : KEY_EMPTY;
-#ifndef FROG_LEAN_REGISTER_MERGE
-    if (EPL >= 8) return (int)merge_inplace<EPL>(S.pool, key, ef_s, lane);      // pools of 256 and 512 keys
-#endif
     return (int)merge_batch<EPL, true>(S.pool, key, ef_s, lane);
 }
 
@@ -184,12 +157,40 @@ __device__ __noinline__ int lean_merge_cold(unsigned char* base, int ns, int ef_
     return lean_merge<EPL, ROWB>(S, ns, ef_s, new_flag, off, lane_id());
 }
 
-template <int EPL, int ROWB>
-#ifdef FROG_LEAN_REGISTER_MERGE
+// Visited check of the cnt <= 64 ranks in en[] (EN order): survivors are compacted, in order, into
+// cand[]; returns their number.  Lane l looks after en[l] and en[l + 32].  With `table` the set is the
+// warp's hash table (L2-resident), otherwise its bitmap slab.
+__device__ __forceinline__ int lean_visit_list(const uint32_t* en, int cnt, uint32_t* cand, uint32_t* table, int table_bits,
+                                               uint32_t* bitmap, uint64_t policy, uint32_t* timeout, int lane) {
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    const bool ha = lane < cnt, hb = lane + 32 < cnt;
+    const uint32_t va = ha ? en[lane] : 0u, vb = hb ? en[lane + 32] : 0u;
+    bool fa, fb;
+    if (table) {
+        if (!table_insert2(table, table_bits, va, ha, vb, hb, fa, fb, policy)) *timeout = 1u;
+    } else {
+        const uint32_t bit_a = 1u << (va & 31), bit_b = 1u << (vb & 31);
+        uint32_t old_a = 0xFFFFFFFFu, old_b = 0xFFFFFFFFu;
+        if (ha) old_a = atomic_or_l2(bitmap + (va >> 5), bit_a, policy);
+        if (hb) old_b = atomic_or_l2(bitmap + (vb >> 5), bit_b, policy);
+        fa = (old_a & bit_a) == 0;
+        fb = (old_b & bit_b) == 0;
+    }
+    const uint32_t Ka = __ballot_sync(FULL, fa), Kb = __ballot_sync(FULL, fb);
+    const int na = __popc(Ka);
+    if (fa) cand[__popc(Ka & lt_mask)] = va;
+    if (fb) cand[na + __popc(Kb & lt_mask)] = vb;
+    __syncwarp();
+    return na + __popc(Kb);
+}
+
+// TABLE: the visited set of a query is a hash table of ranks in global scratch (A.table, 1 << table_bits
+// slots per warp: 16 KB, so that the tables of all resident warps stay in L2 and the test-and-set of a
+// candidate costs no DRAM access; the bitmap's scattered read-modify-writes are what keeps DRAM from the
+// row gathers on large indexes).  The table is exact; a query that fills it half way moves its entries
+// to the warp's bitmap slab and carries on there.
+template <int EPL, int ROWB, bool TABLE>
 __global__ void __launch_bounds__(LEAN_WARPS * 32, EPL <= 4 ? FROG_LEAN_MINB : EPL == 8 ? 12 : 10)
-#else
-__global__ void __launch_bounds__(LEAN_WARPS * 32, FROG_LEAN_MINB)
-#endif
 frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
     using L = Lean<EPL, ROWB>;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -208,15 +209,12 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
     long long t_ph[8] = {0, 0, 0, 0, 0, 0, 0, 0};           // set-up, ENC+visited, gather, merge, output, idle, expansions
     long long t_mark = clock64();
 #endif
-    uint32_t* bitmap = A.bitmap + (size_t)(blockIdx.x * LEAN_WARPS + warp) * A.slab_stride;
+    const size_t warp_id = (size_t)(blockIdx.x * LEAN_WARPS + warp);
+    uint32_t* bitmap = A.bitmap + warp_id * A.slab_stride;
+    uint32_t* const my_table = TABLE ? A.table + (warp_id << A.table_bits) : nullptr;
+    uint32_t* en = reinterpret_cast<uint32_t*>(S.d2);        // admitted ENs of an expansion (the distances come later)
     const uint32_t lt_mask = (1u << lane) - 1u;
-#if defined(FROG_LEAN_SLAB_POLICY) && FROG_LEAN_SLAB_POLICY == 1
-    const uint64_t keep_in_l2 = l2_policy_evict_normal();
-#elif defined(FROG_LEAN_SLAB_POLICY) && FROG_LEAN_SLAB_POLICY == 2
-    const uint64_t keep_in_l2 = l2_policy_evict_first();
-#else
-    const uint64_t keep_in_l2 = l2_policy_evict_last();      // for the visited slab of the running query
-#endif
+    const uint64_t keep_in_l2 = l2_policy_evict_last();      // for the visited set of the running query
 
     for (;;) {
         int q = 0;
@@ -262,9 +260,12 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
                 __syncwarp();
             }
         } else {
-            // visited slab: all-zero here (slab_clean) or zeroed now; see frog_search.cu
+            // Visited set.  TABLE: the warp's hash table (empty here), until the query outgrows it.
+            // Otherwise the bitmap slab: all-zero here (slab_clean) or zeroed now; see frog_search.cu.
+            uint32_t* table = my_table;
+            int n_seen = 0;                                         // ranks in the table
             int n_logged = -1;
-            {
+            if (!TABLE) {
                 const int w0 = l_q >> 5, w1 = r_q >> 5;
                 if (!A.slab_clean)
                     for (int i = w0 + lane; i <= w1; i += 32) st_u32_l2(bitmap + i, 0u, keep_in_l2);
@@ -279,7 +280,12 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
             __syncwarp();
             // lines 2-5: entry points, passed through the visited set
             int ns;
-            {
+            if (TABLE) {
+                if (lane < A.epn) en[lane] = entry_point(A.seed, (uint32_t)l_q, (uint32_t)r_q, lane);
+                __syncwarp();
+                ns = lean_visit_list(en, A.epn, S.cand, table, A.table_bits, bitmap, keep_in_l2, S.timeout, lane);
+                n_seen = ns;
+            } else {
                 const uint32_t ep = entry_point(A.seed, (uint32_t)l_q, (uint32_t)r_q, lane);
                 bool keep = lane < A.epn;
                 if (keep) {
@@ -306,9 +312,18 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
                 const uint32_t u = key_rank(S.pool[first]);               // line 8
                 __syncwarp();
                 if (lane == 0) S.pool[first] |= 1ull;                     // line 9
+                if (TABLE && table && n_seen + 64 > (1 << (A.table_bits - 1))) {
+                    // the next expansion could take the table past half full: move every rank to the
+                    // bitmap slab (all-zero until now) and carry on there; the slab is zeroed by range at the end
+                    for (int i = lane; i < (1 << A.table_bits); i += 32) {
+                        const uint32_t v = __ldcg(table + i);
+                        if (v != TABLE_EMPTY) atomicOr(bitmap + (v >> 5), 1u << (v & 31));
+                    }
+                    __syncwarp();
+                    table = nullptr;
+                }
                 // line 10, Alg. 4 over rows L_start..L_end of ENC(u), four 32-entry chunks per round
-                // trip, admission under budget B across the chunks in order; lines 12-13: the admitted
-                // lanes test-and-set their visited bits in place, survivors are compacted into cand[]
+                // trip, admission under budget B across the chunks in order
                 const uint32_t* hot = A.enc + ((size_t)u * A.H + L_start) * A.m;
                 int cnt = 0;
                 ns = 0;
@@ -321,44 +336,62 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
                     const bool pred0 = (v0 - (uint32_t)l_q) <= span;
                     const uint32_t M0 = __ballot_sync(FULL, pred0);
                     const int a0 = min(__popc(M0), A.B - cnt);
-                    const bool adm0 = pred0 && __popc(M0 & lt_mask) < a0;
+                    const int rank0 = __popc(M0 & lt_mask);
+                    const bool adm0 = pred0 && rank0 < a0;
                     const int rem1 = A.B - cnt - a0;
                     const bool pred1 = rem1 > 0 && ((v1 - (uint32_t)l_q) <= span);
                     const uint32_t M1 = __ballot_sync(FULL, pred1);
                     const int a1 = min(__popc(M1), rem1);
-                    const bool adm1 = pred1 && __popc(M1 & lt_mask) < a1;
+                    const int rank1 = __popc(M1 & lt_mask);
+                    const bool adm1 = pred1 && rank1 < a1;
                     const int rem2 = rem1 - a1;
                     const bool pred2 = rem2 > 0 && ((v2 - (uint32_t)l_q) <= span);
                     const uint32_t M2 = __ballot_sync(FULL, pred2);
                     const int a2 = min(__popc(M2), rem2);
-                    const bool adm2 = pred2 && __popc(M2 & lt_mask) < a2;
+                    const int rank2 = __popc(M2 & lt_mask);
+                    const bool adm2 = pred2 && rank2 < a2;
                     const int rem3 = rem2 - a2;
                     const bool pred3 = rem3 > 0 && ((v3 - (uint32_t)l_q) <= span);
                     const uint32_t M3 = __ballot_sync(FULL, pred3);
                     const int a3 = min(__popc(M3), rem3);
-                    const bool adm3 = pred3 && __popc(M3 & lt_mask) < a3;
-                    const uint32_t bit0 = 1u << (v0 & 31), bit1 = 1u << (v1 & 31);
-                    const uint32_t bit2 = 1u << (v2 & 31), bit3 = 1u << (v3 & 31);
-                    uint32_t old0 = 0xFFFFFFFFu, old1 = 0xFFFFFFFFu, old2 = 0xFFFFFFFFu, old3 = 0xFFFFFFFFu;
-                    if (adm0) old0 = atomic_or_l2(bitmap + (v0 >> 5), bit0, keep_in_l2);
-                    if (adm1) old1 = atomic_or_l2(bitmap + (v1 >> 5), bit1, keep_in_l2);
-                    if (adm2) old2 = atomic_or_l2(bitmap + (v2 >> 5), bit2, keep_in_l2);
-                    if (adm3) old3 = atomic_or_l2(bitmap + (v3 >> 5), bit3, keep_in_l2);
-                    const bool keep0 = (old0 & bit0) == 0, keep1 = (old1 & bit1) == 0;
-                    const bool keep2 = (old2 & bit2) == 0, keep3 = (old3 & bit3) == 0;
-                    const uint32_t K0 = __ballot_sync(FULL, keep0);
-                    const uint32_t K1 = __ballot_sync(FULL, keep1);
-                    const uint32_t K2 = __ballot_sync(FULL, keep2);
-                    const uint32_t K3 = __ballot_sync(FULL, keep3);
-                    const int n0 = __popc(K0), n1 = __popc(K1), n2 = __popc(K2);
-                    if (keep0) S.cand[ns + __popc(K0 & lt_mask)] = v0;
-                    if (keep1) S.cand[ns + n0 + __popc(K1 & lt_mask)] = v1;
-                    if (keep2) S.cand[ns + n0 + n1 + __popc(K2 & lt_mask)] = v2;
-                    if (keep3) S.cand[ns + n0 + n1 + n2 + __popc(K3 & lt_mask)] = v3;
-                    ns += n0 + n1 + n2 + __popc(K3);
+                    const int rank3 = __popc(M3 & lt_mask);
+                    const bool adm3 = pred3 && rank3 < a3;
+                    if (TABLE) {
+                        // lines 12-13 come after the scan: the admitted ENs are listed in order first
+                        if (adm0) en[cnt + rank0] = v0;
+                        if (adm1) en[cnt + a0 + rank1] = v1;
+                        if (adm2) en[cnt + a0 + a1 + rank2] = v2;
+                        if (adm3) en[cnt + a0 + a1 + a2 + rank3] = v3;
+                    } else {
+                        // lines 12-13: the admitted lanes test-and-set their visited bits in place,
+                        // survivors are compacted into cand[]
+                        const uint32_t bit0 = 1u << (v0 & 31), bit1 = 1u << (v1 & 31);
+                        const uint32_t bit2 = 1u << (v2 & 31), bit3 = 1u << (v3 & 31);
+                        uint32_t old0 = 0xFFFFFFFFu, old1 = 0xFFFFFFFFu, old2 = 0xFFFFFFFFu, old3 = 0xFFFFFFFFu;
+                        if (adm0) old0 = atomic_or_l2(bitmap + (v0 >> 5), bit0, keep_in_l2);
+                        if (adm1) old1 = atomic_or_l2(bitmap + (v1 >> 5), bit1, keep_in_l2);
+                        if (adm2) old2 = atomic_or_l2(bitmap + (v2 >> 5), bit2, keep_in_l2);
+                        if (adm3) old3 = atomic_or_l2(bitmap + (v3 >> 5), bit3, keep_in_l2);
+                        const bool keep0 = (old0 & bit0) == 0, keep1 = (old1 & bit1) == 0;
+                        const bool keep2 = (old2 & bit2) == 0, keep3 = (old3 & bit3) == 0;
+                        const uint32_t K0 = __ballot_sync(FULL, keep0);
+                        const uint32_t K1 = __ballot_sync(FULL, keep1);
+                        const uint32_t K2 = __ballot_sync(FULL, keep2);
+                        const uint32_t K3 = __ballot_sync(FULL, keep3);
+                        const int n0 = __popc(K0), n1 = __popc(K1), n2 = __popc(K2);
+                        if (keep0) S.cand[ns + __popc(K0 & lt_mask)] = v0;
+                        if (keep1) S.cand[ns + n0 + __popc(K1 & lt_mask)] = v1;
+                        if (keep2) S.cand[ns + n0 + n1 + __popc(K2 & lt_mask)] = v2;
+                        if (keep3) S.cand[ns + n0 + n1 + n2 + __popc(K3 & lt_mask)] = v3;
+                        ns += n0 + n1 + n2 + __popc(K3);
+                    }
                     cnt += a0 + a1 + a2 + a3;
                 }
                 __syncwarp();
+                if (TABLE) {
+                    ns = lean_visit_list(en, cnt, S.cand, table, A.table_bits, bitmap, keep_in_l2, S.timeout, lane);
+                    n_seen += ns;
+                }
                 ++n_exp;
                 if (n_logged >= 0) n_logged = log_ranks(bitmap + A.bitmap_words, A.log_cap, n_logged, S.cand, ns, lane);
                 // lines 14-17
@@ -373,7 +406,16 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
                 t_ph[7] += ns;
 #endif
             }
-            if (A.slab_clean) {
+            if (TABLE) {
+                // empty the table again; a query that moved to the slab zeroes the words of its range
+                const uint4 e4 = make_uint4(TABLE_EMPTY, TABLE_EMPTY, TABLE_EMPTY, TABLE_EMPTY);
+                uint4* t4 = reinterpret_cast<uint4*>(my_table);
+                for (int i = lane; i < (1 << (A.table_bits - 2)); i += 32) __stcg(t4 + i, e4);
+                if (!table) {
+                    const int w0 = l_q >> 5, w1 = r_q >> 5;
+                    for (int i = w0 + lane; i <= w1; i += 32) bitmap[i] = 0u;
+                }
+            } else if (A.slab_clean) {
                 // leave the slab all-zero: the words of the logged ranks, or of the whole range
                 if (n_logged >= 0) {
                     const uint32_t* log = bitmap + A.bitmap_words;
@@ -417,13 +459,14 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
 }
 
 template <int ROWB>
-frog_kernel_fn lean_pick(int ef_s, size_t* smem_per_warp) {
-    if (ef_s <= 32) { *smem_per_warp = Lean<1, ROWB>::BYTES; return frog_search_lean_kernel<1, ROWB>; }
-    if (ef_s <= 64) { *smem_per_warp = Lean<2, ROWB>::BYTES; return frog_search_lean_kernel<2, ROWB>; }
-    if (ef_s <= 128) { *smem_per_warp = Lean<4, ROWB>::BYTES; return frog_search_lean_kernel<4, ROWB>; }
-    if (ef_s <= 256) { *smem_per_warp = Lean<8, ROWB>::BYTES; return frog_search_lean_kernel<8, ROWB>; }
+frog_kernel_fn lean_pick(int ef_s, bool table, size_t* smem_per_warp) {
+    if (ef_s <= 32) { *smem_per_warp = Lean<1, ROWB>::BYTES; return table ? frog_search_lean_kernel<1, ROWB, true> : frog_search_lean_kernel<1, ROWB, false>; }
+    if (ef_s <= 64) { *smem_per_warp = Lean<2, ROWB>::BYTES; return table ? frog_search_lean_kernel<2, ROWB, true> : frog_search_lean_kernel<2, ROWB, false>; }
+    if (table) return nullptr;
+    if (ef_s <= 128) { *smem_per_warp = Lean<4, ROWB>::BYTES; return frog_search_lean_kernel<4, ROWB, false>; }
+    if (ef_s <= 256) { *smem_per_warp = Lean<8, ROWB>::BYTES; return frog_search_lean_kernel<8, ROWB, false>; }
     *smem_per_warp = Lean<16, ROWB>::BYTES;
-    return frog_search_lean_kernel<16, ROWB>;
+    return frog_search_lean_kernel<16, ROWB, false>;
 }
 
 }  // namespace
@@ -431,11 +474,12 @@ frog_kernel_fn lean_pick(int ef_s, size_t* smem_per_warp) {
 namespace froghost {
 
 // The lean kernel for this beam width and row size, or null if the shape is not covered (the caller
-// then uses the generic kernel).  Needs the row tensor map and the bitmap visited set.
-frog_kernel_fn lean_kernel(int ef_s, int row_bytes, size_t* smem_per_warp, int* warps_per_cta) {
+// then uses the generic kernel).  Needs the row tensor map and the bitmap visited set.  `table`: the
+// variant whose visited set is the L2-resident hash table (pools of up to 64 keys only).
+frog_kernel_fn lean_kernel(int ef_s, int row_bytes, bool table, size_t* smem_per_warp, int* warps_per_cta) {
     *warps_per_cta = LEAN_WARPS;
-    if (row_bytes == 384) return lean_pick<384>(ef_s, smem_per_warp);
-    if (row_bytes == 512) return lean_pick<512>(ef_s, smem_per_warp);
+    if (row_bytes == 384) return lean_pick<384>(ef_s, table, smem_per_warp);
+    if (row_bytes == 512) return lean_pick<512>(ef_s, table, smem_per_warp);
     return nullptr;
 }
 

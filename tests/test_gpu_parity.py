@@ -321,6 +321,32 @@ def test_row_specialised_kernel_at_every_pool_size(libs, cache_dir, name, n, nq)
         gix.close()
 
 
+@pytest.mark.parametrize("name,n,nq", [("sift", 60_000, 300), ("deep1m", 50_000, 300), ("deep10m", 70_001, 300)])
+def test_visited_hash_table_form(libs, cache_dir, name, n, nq):
+    """The visited set as a hash table of ranks in global scratch (what large indexes get at beam widths
+    up to 64), forced here on small indexes: with the full-size table no query outgrows it; with 256 and
+    64 slots almost every query moves to its bitmap slab part of the way.  Results equal the oracle's
+    and the bitmap form's bit for bit, launch after launch (tables and slabs are left clean)."""
+    from conftest import build_scaled
+    wl, path, ix = build_scaled(libs, cache_dir, name, n, nq)
+    gix = libs.Index.load(path, 0)
+    try:
+        q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
+        for ef, k, B in ((32, 10, 64), (64, 10, 64), (24, 5, 16), (48, 48, 33)):
+            ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef, B=B)
+            for bits in (0, 8, 6, 0):
+                prm = libs.Params(budget=B, debug_flags=8 | (bits << 8))
+                ids, dists = gix.search(q, lo, hi, k, ef, params=prm)
+                torch.cuda.synchronize()
+                assert np.array_equal(ids.cpu().numpy(), ref.ids), (ef, bits)
+                assert np.array_equal(dists.cpu().numpy(), ref.dists), (ef, bits)
+            ids, dists = gix.search(q, lo, hi, k, ef, params=libs.Params(budget=B, visited=libs.VISITED_BITMAP))
+            torch.cuda.synchronize()
+            assert np.array_equal(ids.cpu().numpy(), ref.ids) and np.array_equal(dists.cpu().numpy(), ref.dists)
+    finally:
+        gix.close()
+
+
 def test_odd_dimension(libs, cache_dir):
     rng = np.random.default_rng(2)
     V = rng.standard_normal((3000, 10)).astype(np.float32)
