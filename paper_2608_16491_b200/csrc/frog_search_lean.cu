@@ -27,8 +27,11 @@ constexpr int LEAN_WARPS = 2;      // warps per CTA; they never synchronise with
 #ifndef FROG_LEAN_NSLOT_384
 #define FROG_LEAN_NSLOT_384 2      // quads (4 rows each) in the stage ring for 384-byte rows
 #endif
-#ifndef FROG_LEAN_MINB
-#define FROG_LEAN_MINB 16          // resident CTAs per SM the register allocation aims at (pools up to 128 keys)
+#ifndef FROG_LEAN_MINB_384
+#define FROG_LEAN_MINB_384 18      // resident CTAs per SM the register allocation aims at (pools up to 64 keys):
+#endif                             // 36 warps at 56 registers for 384-byte rows (+3 %), 32 warps at 64 for
+#ifndef FROG_LEAN_MINB_512         // 512-byte rows (36 warps measured 8 % slower there)
+#define FROG_LEAN_MINB_512 16
 #endif
 #ifndef FROG_LEAN_NSLOT_512
 #define FROG_LEAN_NSLOT_512 2      // ... for 512-byte rows
@@ -190,7 +193,7 @@ __device__ __forceinline__ int lean_visit_list(const uint32_t* en, int cnt, uint
 // row gathers on large indexes).  The table is exact; a query that fills it half way moves its entries
 // to the warp's bitmap slab and carries on there.
 template <int EPL, int ROWB, bool TABLE>
-__global__ void __launch_bounds__(LEAN_WARPS * 32, EPL <= 4 ? FROG_LEAN_MINB : EPL == 8 ? 12 : 10)
+__global__ void __launch_bounds__(LEAN_WARPS * 32, EPL <= 2 ? (ROWB <= 384 ? FROG_LEAN_MINB_384 : FROG_LEAN_MINB_512) : EPL == 4 ? 16 : EPL == 8 ? 12 : 10)
 frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
     using L = Lean<EPL, ROWB>;
     extern __shared__ __align__(128) unsigned char smem_raw[];
