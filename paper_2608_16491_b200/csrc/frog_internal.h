@@ -17,6 +17,8 @@ struct FrogScratch {
     size_t bitmap_slots = 0;
     uint32_t* d_table = nullptr;     // table_slots visited hash tables of FROG_TABLE_SLOTS ranks (all 0xFFFFFFFF at rest)
     size_t table_slots = 0;
+    int table_bits = 0;              // log2 of the ranks per table of the last launch
+    size_t table_bytes = 0;
     int32_t* d_plan = nullptr;       // per query: rank interval (2 ints) and processing order (1 int)
     size_t plan_queries = 0;
     cudaEvent_t done = nullptr;
@@ -25,6 +27,7 @@ struct FrogScratch {
 };
 constexpr int FROG_SCRATCH_SETS = 4;
 constexpr int FROG_TABLE_BITS = 12;    // 4,096 ranks = 16 KB per resident warp: 78 MB for a full grid, inside L2
+constexpr int FROG_TABLE_BITS_WIDE = 13;   // beam widths 65..128: 8,192 ranks (a query evaluates ~2,000 there)
 
 struct frog_index {
     frog_index_info_t info;
@@ -100,7 +103,7 @@ int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in
 bool make_row_tensor_map(const void* base, bool f16, int row_elems, size_t row_bytes, size_t n, CUtensorMap* out);
 int acquire_scratch(frog_index* ix, cudaStream_t s, FrogScratch** out);
 int ensure_bitmap(const frog_index* ix, FrogScratch* sc, size_t slots);
-int ensure_table(FrogScratch* sc, size_t slots);
+int ensure_table(FrogScratch* sc, size_t slots, int bits);
 int ensure_plan(FrogScratch* sc, size_t nq);
 }  // namespace froghost
 

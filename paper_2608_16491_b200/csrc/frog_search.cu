@@ -571,7 +571,7 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
         // 4,194,304 objects and more: measured 1.26x faster at 10M objects, 0.85x at 1M, where the bits a
         // query touches still fit L2) and the pool is small enough for a query to fit the table as a rule;
         // FROG_VISITED_BITMAP keeps the bitmap
-        table = allow_table && P.visited == FROG_VISITED_AUTO && beam_width <= 64 &&
+        table = allow_table && P.visited == FROG_VISITED_AUTO && beam_width <= 128 &&
                 (bitmap_words_per_slot(ix) >= (size_t)TABLE_MIN_SLAB_WORDS || (P.debug_flags & 8));
         kernel_fn lean = froghost::lean_kernel(beam_width, ix->info.d_pad * 4, table, &per_warp, &wpc);
         if (!lean && table) {
@@ -758,13 +758,19 @@ int ensure_bitmap(const frog_index* ix, FrogScratch* sc, size_t slots) {
 }
 
 // Visited hash tables for `slots` resident warps, all entries empty (the kernel leaves them so).
-int ensure_table(FrogScratch* sc, size_t slots) {
-    if (sc->d_table && sc->table_slots >= slots) return FROG_OK;
+int ensure_table(FrogScratch* sc, size_t slots, int bits) {
+    // the tables are all-empty at rest, so an allocation can be re-cut into tables of another size
+    const size_t bytes = (slots << bits) * sizeof(uint32_t);
+    if (sc->d_table && sc->table_bytes >= bytes) {
+        sc->table_bits = bits;
+        sc->table_slots = sc->table_bytes / sizeof(uint32_t) >> bits;
+        return FROG_OK;
+    }
     FROG_CUDA_TRY(cudaDeviceSynchronize());
     if (sc->d_table) FROG_CUDA_TRY(cudaFree(sc->d_table));
     sc->d_table = nullptr;
     sc->table_slots = 0;
-    const size_t bytes = (slots << FROG_TABLE_BITS) * sizeof(uint32_t);
+    sc->table_bytes = 0;
     cudaError_t e = cudaMalloc(&sc->d_table, bytes);
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -773,6 +779,8 @@ int ensure_table(FrogScratch* sc, size_t slots) {
     }
     FROG_CUDA_TRY(cudaMemset(sc->d_table, 0xFF, bytes));
     FROG_CUDA_TRY(cudaDeviceSynchronize());
+    sc->table_bytes = bytes;
+    sc->table_bits = bits;
     sc->table_slots = slots;
     return FROG_OK;
 }
@@ -846,7 +854,8 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
         }
         if (rc) return rc;
     }
-    if (plan.table && froghost::ensure_table(sc, (size_t)plan.grid * WARPS_PER_CTA) != FROG_OK) {
+    const int table_bits = beam_width <= 64 ? FROG_TABLE_BITS : FROG_TABLE_BITS_WIDE;
+    if (plan.table && froghost::ensure_table(sc, (size_t)plan.grid * WARPS_PER_CTA, table_bits) != FROG_OK) {
         rc = plan_launch(index, beam_width, P, mode, bitmap, nq, &plan, false);     // no room: bitmap only
         if (rc) return rc;
     }
@@ -887,8 +896,8 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     A.slab_stride = A.bitmap_words + (size_t)A.log_cap;
     A.slab_clean = 1;
     A.table = plan.table ? sc->d_table : nullptr;
-    A.table_bits = FROG_TABLE_BITS;
-    if (((P.debug_flags >> 8) & 15) >= 6 && ((P.debug_flags >> 8) & 15) <= FROG_TABLE_BITS)
+    A.table_bits = table_bits;
+    if (((P.debug_flags >> 8) & 15) >= 6 && ((P.debug_flags >> 8) & 15) <= table_bits)
         A.table_bits = (P.debug_flags >> 8) & 15;           // tests: a small table, so that queries outgrow it
     A.ranges = nullptr;
     A.order = nullptr;

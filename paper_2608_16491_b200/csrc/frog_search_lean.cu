@@ -465,8 +465,8 @@ template <int ROWB>
 frog_kernel_fn lean_pick(int ef_s, bool table, size_t* smem_per_warp) {
     if (ef_s <= 32) { *smem_per_warp = Lean<1, ROWB>::BYTES; return table ? frog_search_lean_kernel<1, ROWB, true> : frog_search_lean_kernel<1, ROWB, false>; }
     if (ef_s <= 64) { *smem_per_warp = Lean<2, ROWB>::BYTES; return table ? frog_search_lean_kernel<2, ROWB, true> : frog_search_lean_kernel<2, ROWB, false>; }
+    if (ef_s <= 128) { *smem_per_warp = Lean<4, ROWB>::BYTES; return table ? frog_search_lean_kernel<4, ROWB, true> : frog_search_lean_kernel<4, ROWB, false>; }
     if (table) return nullptr;
-    if (ef_s <= 128) { *smem_per_warp = Lean<4, ROWB>::BYTES; return frog_search_lean_kernel<4, ROWB, false>; }
     if (ef_s <= 256) { *smem_per_warp = Lean<8, ROWB>::BYTES; return frog_search_lean_kernel<8, ROWB, false>; }
     *smem_per_warp = Lean<16, ROWB>::BYTES;
     return frog_search_lean_kernel<16, ROWB, false>;
@@ -478,7 +478,7 @@ namespace froghost {
 
 // The lean kernel for this beam width and row size, or null if the shape is not covered (the caller
 // then uses the generic kernel).  Needs the row tensor map and the bitmap visited set.  `table`: the
-// variant whose visited set is the L2-resident hash table (pools of up to 64 keys only).
+// variant whose visited set is the L2-resident hash table (pools of up to 128 keys only).
 frog_kernel_fn lean_kernel(int ef_s, int row_bytes, bool table, size_t* smem_per_warp, int* warps_per_cta) {
     *warps_per_cta = LEAN_WARPS;
     if (row_bytes == 384) return lean_pick<384>(ef_s, table, smem_per_warp);
