@@ -74,6 +74,7 @@ typedef struct {
                            bit 2: use the general kernel where a kernel specialised for the row size exists
                                   (same results; for comparing the two);
                            bit 3: use the visited hash table (see FROG_VISITED_AUTO) on small indexes too;
+                           bit 4: record CUDA events around the search kernel alone (frog_search_kernel_ms);
                            bits 8-11: log2 of that table's slots, 6..12 (0 = 12), to make queries outgrow it */
     int32_t exact_below;/* ranges holding at most max(beam_width, exact_below) objects are answered by
                            scanning their contiguous rank slab (exact, status FROG_ST_EXACT) instead of
@@ -219,6 +220,11 @@ int frog_search_host(frog_index_t* index, const float* queries, const int32_t* l
 int frog_search_static(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
                        int nq, int k, int beam_width, const frog_params_t* params,
                        int32_t* out_ids, float* out_dists, void* stream);
+
+/* Device time, in milliseconds, of the search kernel of the last frog_search_ex call on `stream` that
+ * was made with params->debug_flags bit 4 set (the call also runs two small planning kernels, which
+ * this figure leaves out).  Waits for that kernel to finish.  INVALID_ARG if there was no such call. */
+int frog_search_kernel_ms(const frog_index_t* index, void* stream, float* ms);
 
 /* Launch shape of the search kernel for the given beam width (for reporting): CTAs, threads per
  * CTA, dynamic shared memory per CTA, query slots resident per SM. */

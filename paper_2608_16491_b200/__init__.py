@@ -290,6 +290,15 @@ class Index:
             raise FrogError(rc, "frog_search_host")
         return out_ids, out_dists
 
+    def kernel_ms(self, stream=None) -> float:
+        """Device time of the search kernel of the last search on ``stream`` made with
+        ``Params(debug_flags=16)`` (waits for it)."""
+        ms = C.c_float()
+        rc = _lib.frog_search_kernel_ms(self._h, _stream_ptr(stream), C.byref(ms))
+        if rc:
+            raise FrogError(rc, "frog_search_kernel_ms")
+        return float(ms.value)
+
     def launch_info(self, beam_width: int, params: Optional[Params] = None):
         g, b, s, qsm = C.c_int(), C.c_int(), C.c_int(), C.c_int()
         rc = _lib.frog_search_launch_info(self._h, C.c_int(beam_width),

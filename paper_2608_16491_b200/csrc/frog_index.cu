@@ -118,6 +118,8 @@ extern "C" void frog_index_free(frog_index_t* ix) {
             cudaFree(ix->scratch[i].d_table);
             cudaFree(ix->scratch[i].d_plan);
             if (ix->scratch[i].done) cudaEventDestroy(ix->scratch[i].done);
+            if (ix->scratch[i].k_begin) cudaEventDestroy(ix->scratch[i].k_begin);
+            if (ix->scratch[i].k_end) cudaEventDestroy(ix->scratch[i].k_end);
         }
         cudaFree(ix->d_stage);
     }

@@ -22,6 +22,8 @@ struct FrogScratch {
     int32_t* d_plan = nullptr;       // per query: rank interval (2 ints) and processing order (1 int)
     size_t plan_queries = 0;
     cudaEvent_t done = nullptr;
+    cudaEvent_t k_begin = nullptr, k_end = nullptr;   // around the search kernel of the last timed launch
+    bool k_timed = false;
     cudaStream_t stream = nullptr;   // stream of the last launch
     unsigned long long tick = 0;
 };

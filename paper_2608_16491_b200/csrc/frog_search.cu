@@ -914,12 +914,36 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
         A.ranges = ranges;
         A.order = order;
     }
+    const bool timed = (P.debug_flags & 16) != 0;          // events around the search kernel alone
+    if (timed) {
+        if (!sc->k_begin) FROG_CUDA_TRY(cudaEventCreate(&sc->k_begin));
+        if (!sc->k_end) FROG_CUDA_TRY(cudaEventCreate(&sc->k_end));
+        FROG_CUDA_TRY(cudaEventRecord(sc->k_begin, s));
+    }
     plan.fn<<<plan.grid, plan.block, plan.smem, s>>>(A);
     FROG_CUDA_TRY(cudaGetLastError());
+    if (timed) FROG_CUDA_TRY(cudaEventRecord(sc->k_end, s));
+    sc->k_timed = timed;
     FROG_CUDA_TRY(cudaEventRecord(sc->done, s));
     sc->stream = s;
     sc->tick = ++mix->tick;
     return FROG_OK;
+}
+
+extern "C" int frog_search_kernel_ms(const frog_index_t* index, void* stream, float* ms) {
+    if (!index || !ms) return FROG_ERR_INVALID_ARG;
+    frog_index* mix = const_cast<frog_index*>(index);
+    std::lock_guard<std::mutex> lock(mix->mu);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < mix->n_scratch; ++i) {
+        FrogScratch& sc = mix->scratch[i];
+        if (sc.tick && sc.stream == s && sc.k_timed) {
+            FROG_CUDA_TRY(cudaEventSynchronize(sc.k_end));
+            FROG_CUDA_TRY(cudaEventElapsedTime(ms, sc.k_begin, sc.k_end));
+            return FROG_OK;
+        }
+    }
+    return FROG_ERR_INVALID_ARG;           // no timed launch on this stream
 }
 
 extern "C" int frog_search(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
