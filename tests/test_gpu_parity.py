@@ -205,6 +205,31 @@ def test_small_visited_table_changes_work_not_results(libs, tiny_gpu):
     assert (got[2] & 16).any()
 
 
+def test_search_kernel_time_is_reported_on_request(libs, tiny_gpu):
+    """debug_flags bit 4 makes the call record events around the search kernel alone; the time read
+    back is positive and no longer than the whole call (two planning kernels included) as timed by
+    events on the same stream; without the flag there is nothing to read."""
+    wl, ix, gix = tiny_gpu
+    q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
+    side = torch.cuda.Stream()
+    with pytest.raises(libs.FrogError):
+        gix.kernel_ms(stream=side)                         # no timed launch on this stream yet
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    gix.search(q, lo, hi, wl.k, 64, params=libs.Params(debug_flags=16), stream=side)    # warm
+    side.synchronize()
+    e0.record(side)
+    ids, _ = gix.search(q, lo, hi, wl.k, 64, params=libs.Params(debug_flags=16), stream=side)
+    e1.record(side)
+    ms = gix.kernel_ms(stream=side)
+    side.synchronize()
+    assert 0.0 < ms <= e0.elapsed_time(e1) * 1.05
+    ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, 64)
+    assert np.array_equal(ids.cpu().numpy(), ref.ids)
+    gix.search(q, lo, hi, wl.k, 64, stream=side)            # an untimed launch on the same stream
+    with pytest.raises(libs.FrogError):
+        gix.kernel_ms(stream=side)
+
+
 def test_empty_batch_and_argument_errors(libs, tiny_gpu):
     wl, ix, gix = tiny_gpu
     q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
