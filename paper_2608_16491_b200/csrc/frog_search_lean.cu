@@ -1,21 +1,24 @@
-// The search kernel for the common case, trimmed for instruction count: fp32 rows of 384 or 512
-// bytes (d = 96, 128), exact (bitmap) visited set, rows fetched four at a time by the copy engine's
-// tile::gather4, no counters and no trace.  It computes exactly what frog_search_kernel computes
-// (paper Alg. 2 with Alg. 3 once per query and Alg. 4 + the lazy hash check per expansion; same
-// distance order, same merge), and the tests compare the two bit for bit.
+// The search kernel for the common case: fp32 rows of 384 or 512 bytes (d = 96, 128), an exact
+// visited set in global scratch (bitmap slab, or for large indexes a hash table of ranks), rows
+// fetched four at a time by the copy engine's tile::gather4, no counters and no trace.  It
+// computes exactly what frog_search_kernel computes (paper Alg. 2 with Alg. 3 once per query and
+// Alg. 4 + the lazy hash check per expansion; same distance order, same merge), and the tests
+// compare the two bit for bit.
 //
-// Why a second kernel: with short rows the generic kernel spends ~960 warp instructions per
-// expansion for ~12 distance evaluations and keeps 68 % of the issue slots busy -- it is bound by
-// instruction issue and dependent latency, not by bytes.  Here
-//   * the stage buffer is a ring of NSLOT quads (4 rows each, one mbarrier per quad): 12 rows of
-//     384 bytes are in flight per warp instead of 8, and lane 0 issues every copy of an expansion
-//     from one short loop (the rank list is padded to a whole quad with rows beyond the tensor,
-//     which arrive as zeros, so a copy needs no per-row selects);
+// Why a second kernel: with short rows the general kernel spends 1,000-1,400 warp instructions per
+// expansion for 10-20 distance evaluations and keeps 60-70 % of the issue slots busy -- it is bound
+// by instruction issue and dependent latency, not by bytes.  Here
+//   * the stage buffer is a ring of two quads (4 rows each, one mbarrier per quad) and lane 0
+//     issues the copies from one short block (the rank list is padded to a whole quad with rows
+//     beyond the tensor, which arrive as zeros, so a copy needs no per-row selects); deeper rings
+//     were measured slower;
 //   * a team's leader stores its row's squared distance to shared memory, every lane picks up
 //     "its" distance with one load (no shuffle/compare chain to route results to lanes);
 //   * up to 64 survivors of one expansion go through one gather loop;
 //   * everything in the expansion loop is inlined (no call, no argument shuffling), the row
-//     geometry and the shared-memory layout are compile-time constants.
+//     geometry and the shared-memory layout are compile-time constants;
+//   * on indexes of 4M objects and more the visited set is a 16 KB hash table per warp that stays
+//     in L2 instead of a bitmap slab of n/8 bytes per warp that does not.
 #include "frog_device.cuh"
 #include "frog_internal.h"
 
