@@ -221,6 +221,13 @@ int frog_search_static(const frog_index_t* index, const float* queries, const in
                        int nq, int k, int beam_width, const frog_params_t* params,
                        int32_t* out_ids, float* out_dists, void* stream);
 
+/* FROG_ST_* conditions of the last frog_search / frog_search_ex / frog_search_host launch on `stream`
+ * that concern the whole launch rather than one query: today FROG_ST_COPY_TIMEOUT (some row of the
+ * result was written as padding because a bulk copy never completed; never expected).  Lets a caller
+ * that passes no `status` array notice it.  Waits for that launch to finish.  INVALID_ARG if there
+ * was no launch on the stream.  frog_search_static keeps no such word. */
+int frog_search_last_status(const frog_index_t* index, void* stream, uint32_t* flags);
+
 /* Device time, in milliseconds, of the search kernel of the last frog_search_ex call on `stream` that
  * was made with params->debug_flags bit 4 set (the call also runs two small planning kernels, which
  * this figure leaves out).  Waits for that kernel to finish.  INVALID_ARG if there was no such call. */

@@ -290,6 +290,14 @@ class Index:
             raise FrogError(rc, "frog_search_host")
         return out_ids, out_dists
 
+    def last_status(self, stream=None) -> int:
+        """Launch-wide FROG_ST_* bits of the last search on ``stream`` (0 = nothing to report)."""
+        flags = C.c_uint32()
+        rc = _lib.frog_search_last_status(self._h, _stream_ptr(stream), C.byref(flags))
+        if rc:
+            raise FrogError(rc, "frog_search_last_status")
+        return int(flags.value)
+
     def kernel_ms(self, stream=None) -> float:
         """Device time of the search kernel of the last search on ``stream`` made with
         ``Params(debug_flags=16)`` (waits for it)."""

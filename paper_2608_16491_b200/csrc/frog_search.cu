@@ -440,6 +440,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
         if (got < A.k) st |= FROG_ST_SHORT;
         if (__any_sync(FULL, forgets != 0)) st |= FROG_ST_FORGOT;   // counted per lane
         if (bad) st |= FROG_ST_COPY_TIMEOUT;
+        if (bad && lane == 0) atomicOr(A.work_counter + 1, FROG_ST_COPY_TIMEOUT);   // sticky word of this launch
         FROG_PHASE(4);
         if (lane == 0) {
             if (A.status) A.status[q] = st;
@@ -928,6 +929,24 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     sc->stream = s;
     sc->tick = ++mix->tick;
     return FROG_OK;
+}
+
+extern "C" int frog_search_last_status(const frog_index_t* index, void* stream, uint32_t* flags) {
+    if (!index || !flags) return FROG_ERR_INVALID_ARG;
+    frog_index* mix = const_cast<frog_index*>(index);
+    std::lock_guard<std::mutex> lock(mix->mu);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < mix->n_scratch; ++i) {
+        FrogScratch& sc = mix->scratch[i];
+        if (sc.tick && sc.stream == s) {
+            FROG_CUDA_TRY(cudaEventSynchronize(sc.done));
+            unsigned int word = 0;
+            FROG_CUDA_TRY(cudaMemcpy(&word, sc.d_work + 1, sizeof(word), cudaMemcpyDeviceToHost));
+            *flags = word;
+            return FROG_OK;
+        }
+    }
+    return FROG_ERR_INVALID_ARG;           // no launch on this stream
 }
 
 extern "C" int frog_search_kernel_ms(const frog_index_t* index, void* stream, float* ms) {

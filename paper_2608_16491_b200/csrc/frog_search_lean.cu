@@ -449,6 +449,7 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
             A.out_ids[(size_t)q * A.k + j] = oid;
             A.out_dists[(size_t)q * A.k + j] = dist;
         }
+        if (bad && lane == 0) atomicOr(A.work_counter + 1, FROG_ST_COPY_TIMEOUT);   // sticky word of this launch
         if (A.status) {
             got = __reduce_add_sync(FULL, got);
             if (got < A.k) st |= FROG_ST_SHORT;

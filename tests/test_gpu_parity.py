@@ -228,6 +228,10 @@ def test_search_kernel_time_is_reported_on_request(libs, tiny_gpu):
     gix.search(q, lo, hi, wl.k, 64, stream=side)            # an untimed launch on the same stream
     with pytest.raises(libs.FrogError):
         gix.kernel_ms(stream=side)
+    # the launch-wide status word: nothing to report after a normal launch; unknown streams are refused
+    assert gix.last_status(stream=side) == 0
+    with pytest.raises(libs.FrogError):
+        gix.last_status(stream=torch.cuda.Stream())
 
 
 def test_empty_batch_and_argument_errors(libs, tiny_gpu):
