@@ -36,6 +36,13 @@ constexpr int LEAN_WARPS = 2;      // warps per CTA; they never synchronise with
 #ifndef FROG_LEAN_MINB_512         // 512-byte rows (36 warps measured 8 % slower there)
 #define FROG_LEAN_MINB_512 16
 #endif
+#ifndef FROG_LEAN_MINB_POOL256
+#define FROG_LEAN_MINB_POOL256 14  // pools of 256 keys: 72 registers, 28 warps (the merge holds 8 keys per lane;
+                                   // measured +3-4 % over 24 warps at 80 registers, 32 warps at 64: +1-2 %)
+#endif
+#ifndef FROG_LEAN_MINB_POOL512
+#define FROG_LEAN_MINB_POOL512 10  // pools of 512 keys: 96 registers
+#endif
 #ifndef FROG_LEAN_NSLOT_512
 #define FROG_LEAN_NSLOT_512 2      // ... for 512-byte rows
 #endif
@@ -196,7 +203,7 @@ __device__ __forceinline__ int lean_visit_list(const uint32_t* en, int cnt, uint
 // row gathers on large indexes).  The table is exact; a query that fills it half way moves its entries
 // to the warp's bitmap slab and carries on there.
 template <int EPL, int ROWB, bool TABLE>
-__global__ void __launch_bounds__(LEAN_WARPS * 32, EPL <= 2 ? (ROWB <= 384 ? FROG_LEAN_MINB_384 : FROG_LEAN_MINB_512) : EPL == 4 ? 16 : EPL == 8 ? 12 : 10)
+__global__ void __launch_bounds__(LEAN_WARPS * 32, EPL <= 2 ? (ROWB <= 384 ? FROG_LEAN_MINB_384 : FROG_LEAN_MINB_512) : EPL == 4 ? 16 : EPL == 8 ? FROG_LEAN_MINB_POOL256 : FROG_LEAN_MINB_POOL512)
 frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
     using L = Lean<EPL, ROWB>;
     extern __shared__ __align__(128) unsigned char smem_raw[];
