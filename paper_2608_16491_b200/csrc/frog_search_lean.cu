@@ -27,25 +27,50 @@ using namespace frogdev;
 namespace {
 
 constexpr int LEAN_WARPS = 2;      // warps per CTA; they never synchronise with each other
+// Tuning constants (overridable for scratch builds).  NSLOT: quads (4 rows each) in the stage ring.
+// MINB: resident CTAs per SM that the register allocation aims at, per row size and pool size; the
+// values are the measured optima.  More than about 100 KB of tensor copies in flight per SM makes
+// the copy engine's throughput fall off, which is why 512-byte rows want fewer warps than 384-byte
+// rows once the registers of a larger pool cost occupancy anyway.
 #ifndef FROG_LEAN_NSLOT_384
-#define FROG_LEAN_NSLOT_384 2      // quads (4 rows each) in the stage ring for 384-byte rows
-#endif
-#ifndef FROG_LEAN_MINB_384
-#define FROG_LEAN_MINB_384 18      // resident CTAs per SM the register allocation aims at (pools up to 64 keys):
-#endif                             // 36 warps at 56 registers for 384-byte rows (+3 %), 32 warps at 64 for
-#ifndef FROG_LEAN_MINB_512         // 512-byte rows (36 warps measured 8 % slower there)
-#define FROG_LEAN_MINB_512 16
-#endif
-#ifndef FROG_LEAN_MINB_POOL256
-#define FROG_LEAN_MINB_POOL256 14  // pools of 256 keys: 72 registers, 28 warps (the merge holds 8 keys per lane;
-                                   // measured +3-4 % over 24 warps at 80 registers, 32 warps at 64: +1-2 %)
-#endif
-#ifndef FROG_LEAN_MINB_POOL512
-#define FROG_LEAN_MINB_POOL512 10  // pools of 512 keys: 96 registers
+#define FROG_LEAN_NSLOT_384 2
 #endif
 #ifndef FROG_LEAN_NSLOT_512
-#define FROG_LEAN_NSLOT_512 2      // ... for 512-byte rows
+#define FROG_LEAN_NSLOT_512 2
 #endif
+#ifndef FROG_LEAN_MINB_384
+#define FROG_LEAN_MINB_384 18       // 384-byte rows, pools of 32 and 64 keys: 36 warps at 56 registers (+3 % over 32)
+#endif
+#ifndef FROG_LEAN_MINB_384_P128
+#define FROG_LEAN_MINB_384_P128 16  // ... 128 keys: 32 warps (56 registers spill there; 28 and 24 warps: 5-12 % slower)
+#endif
+#ifndef FROG_LEAN_MINB_POOL192
+#define FROG_LEAN_MINB_POOL192 16   // ... 192 keys (beams 129-192): 32 warps at 64 registers (28: -2 %, 24: -5 %)
+#endif
+#ifndef FROG_LEAN_MINB_POOL256
+#define FROG_LEAN_MINB_POOL256 14   // ... 256 keys: 28 warps at 72 registers (the merge holds 8 keys per lane;
+#endif                              // +3-4 % over 24 warps at 80 registers, 32 warps at 64: +1-2 %)
+#ifndef FROG_LEAN_MINB_POOL512
+#define FROG_LEAN_MINB_POOL512 10   // pools of 512 keys, both row sizes: 20 warps at 96 registers (16 and 24: slower)
+#endif
+#ifndef FROG_LEAN_MINB_512
+#define FROG_LEAN_MINB_512 16       // 512-byte rows, pools of 32 and 64 keys: 32 warps (36: 8 % slower, 28 and 24: 1-2 % slower)
+#endif
+#ifndef FROG_LEAN_MINB_512_P128
+#define FROG_LEAN_MINB_512_P128 12  // ... 128 keys: 24 warps (+12 % over 32)
+#endif
+#ifndef FROG_LEAN_MINB_512_P192
+#define FROG_LEAN_MINB_512_P192 12  // ... 192 keys: 24 warps (28 and 20: 11 % slower)
+#endif
+#ifndef FROG_LEAN_MINB_512_P256
+#define FROG_LEAN_MINB_512_P256 12  // ... 256 keys: 24 warps (+12 % over 28)
+#endif
+__host__ __device__ constexpr int lean_min_ctas(int epl, int rowb) {
+    return rowb <= 384 ? (epl <= 2 ? FROG_LEAN_MINB_384 : epl == 4 ? FROG_LEAN_MINB_384_P128 : epl == 6 ? FROG_LEAN_MINB_POOL192
+                          : epl == 8 ? FROG_LEAN_MINB_POOL256 : FROG_LEAN_MINB_POOL512)
+                       : (epl <= 2 ? FROG_LEAN_MINB_512 : epl == 4 ? FROG_LEAN_MINB_512_P128 : epl == 6 ? FROG_LEAN_MINB_512_P192
+                          : epl == 8 ? FROG_LEAN_MINB_512_P256 : FROG_LEAN_MINB_POOL512);
+}
 
 // Scratch builds with -DFROG_LEAN_PROFILE add per-phase cycle counters (summed over all warps into
 // g_lean_prof, read back through frog_debug_lean_profile); the shipped library has none of this.
@@ -203,7 +228,7 @@ __device__ __forceinline__ int lean_visit_list(const uint32_t* en, int cnt, uint
 // row gathers on large indexes).  The table is exact; a query that fills it half way moves its entries
 // to the warp's bitmap slab and carries on there.
 template <int EPL, int ROWB, bool TABLE>
-__global__ void __launch_bounds__(LEAN_WARPS * 32, EPL <= 2 ? (ROWB <= 384 ? FROG_LEAN_MINB_384 : FROG_LEAN_MINB_512) : EPL == 4 ? 16 : EPL == 8 ? FROG_LEAN_MINB_POOL256 : FROG_LEAN_MINB_POOL512)
+__global__ void __launch_bounds__(LEAN_WARPS * 32, lean_min_ctas(EPL, ROWB))
 frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
     using L = Lean<EPL, ROWB>;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -478,6 +503,7 @@ frog_kernel_fn lean_pick(int ef_s, bool table, size_t* smem_per_warp) {
     if (ef_s <= 64) { *smem_per_warp = Lean<2, ROWB>::BYTES; return table ? frog_search_lean_kernel<2, ROWB, true> : frog_search_lean_kernel<2, ROWB, false>; }
     if (ef_s <= 128) { *smem_per_warp = Lean<4, ROWB>::BYTES; return table ? frog_search_lean_kernel<4, ROWB, true> : frog_search_lean_kernel<4, ROWB, false>; }
     if (table) return nullptr;
+    if (ef_s <= 192) { *smem_per_warp = Lean<6, ROWB>::BYTES; return frog_search_lean_kernel<6, ROWB, false>; }
     if (ef_s <= 256) { *smem_per_warp = Lean<8, ROWB>::BYTES; return frog_search_lean_kernel<8, ROWB, false>; }
     *smem_per_warp = Lean<16, ROWB>::BYTES;
     return frog_search_lean_kernel<16, ROWB, false>;

@@ -326,7 +326,7 @@ def test_scaled_workloads_match_oracle(libs, cache_dir, name, n, nq):
 @pytest.mark.parametrize("name,n,nq", [("sift", 60_000, 300), ("deep1m", 50_000, 300)])
 def test_row_specialised_kernel_at_every_pool_size(libs, cache_dir, name, n, nq):
     """Rows of 512 and 384 bytes are searched by a kernel specialised for them (every pool size from
-    32 to 512 keys is its own instantiation).  The plain call (which takes it) against the oracle and,
+    32 to 512 keys — 32, 64, 128, 192, 256, 512 — is its own instantiation).  The plain call (which takes it) against the oracle and,
     inside _gpu_search, against the counting variant of the general kernel, bit for bit; then the
     general kernel forced by debug_flags bit 2 against the same reference."""
     from conftest import build_scaled
@@ -334,7 +334,7 @@ def test_row_specialised_kernel_at_every_pool_size(libs, cache_dir, name, n, nq)
     gix = libs.Index.load(path, 0)
     try:
         for ef, k, kw in ((24, 10, dict(budget=64)), (64, 64, dict(budget=64, epn=32)), (128, 10, dict(budget=64)),
-                          (200, 100, dict(budget=48)), (256, 10, dict(budget=64, max_iters=40)),
+                          (176, 10, dict(budget=64)), (200, 100, dict(budget=48)), (256, 10, dict(budget=64, max_iters=40)),
                           (512, 10, dict(budget=64)), (96, 10, dict(budget=64, exact_below=2000)),
                           (40, 10, dict(budget=64, no_hotspot=1, seed=9))):
             ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef, epn=kw.get("epn", 16), B=kw["budget"],
