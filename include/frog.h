@@ -41,7 +41,7 @@ enum {
 
 /* Limits of the search kernels. */
 #define FROG_MAX_BEAM_WIDTH 512 /* ef_s */
-#define FROG_MAX_BUDGET 64      /* expansion budget B */
+#define FROG_MAX_BUDGET 128     /* expansion budget B */
 #define FROG_MAX_EPN 32         /* entry points */
 
 typedef struct {
@@ -62,7 +62,7 @@ typedef struct {
 /* Optional query-time parameters (Alg. 2 arguments other than k and ef_s). */
 typedef struct {
     int32_t epn;        /* entry points, 1..32; 0 = default 16 (paper Sec. 8.1.4) */
-    int32_t budget;     /* expansion budget B, 1..64; 0 = default 16 */
+    int32_t budget;     /* expansion budget B, 1..128; 0 = default 16 */
     int32_t max_iters;  /* hard cap on expansions per query; 0 = default 16 * beam_width */
     int32_t no_hotspot; /* nonzero: scan all H layers instead of the hotspot (ablation) */
     uint64_t seed;      /* seed of the entry-point generator */
@@ -167,8 +167,8 @@ int frog_search(const frog_index_t* index, const float* queries, const int32_t* 
  *           by Alg. 4, distance evaluations}.  Asking for them selects a variant of the kernel
  *           that keeps these counters (a few per cent slower than the plain one; same results)
  *   trace   DEVICE nq x trace_cap uint32 or null: row q = [len, then per expansion
- *           u, |EN(u)|, EN(u)[0..]] (ranks); records are appended while at least 66 words
- *           remain in the row.  Selects a slower kernel instantiation; meant for tests. */
+ *           u, |EN(u)|, EN(u)[0..]] (ranks); records are appended while at least 2 + max(64, B)
+ *           words remain in the row.  Selects a slower kernel instantiation; meant for tests. */
 int frog_search_ex(const frog_index_t* index, const float* queries, const int32_t* lo, const int32_t* hi,
                    int nq, int k, int beam_width, const frog_params_t* params,
                    int32_t* out_ids, float* out_dists, uint32_t* status, uint32_t* stats,

@@ -351,7 +351,7 @@ void search_one(const Index& ix, const float* v_q, int32_t lo, int32_t hi, int k
                 : en_identification(ix.enc + (int64_t)u * ix.H * ix.m, ix.m, l_q, r_q,
                                     L_start, L_end, P.B, P.warp, EN.data(), &rows);       // line 10
             ++n_exp; n_rows += rows; n_en += cnt;
-            if (trace && trace_ok && (int64_t)trace->size() + 66 > trace_cap - 1) trace_ok = false;   // 66 = header + 64 entries
+            if (trace && trace_ok && (int64_t)trace->size() + 2 + std::max(64, P.B) > trace_cap - 1) trace_ok = false;   // room for a full record
             if (trace && trace_ok) {
                 trace->push_back(u);
                 trace->push_back((uint32_t)cnt);

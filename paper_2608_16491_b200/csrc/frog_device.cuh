@@ -636,13 +636,12 @@ __device__ __forceinline__ uint32_t entry_point(unsigned long long seed, uint32_
 // zero only those words afterwards; narrower ones zero the words of the range (<= 32 KB).
 constexpr int SPARSE_MIN_WORDS = 8192;
 
-// Append the ns <= 64 ranks of cand[] (the vertices whose visited bit this query has just set) to the
+// Append the ns <= 128 ranks of cand[] (the vertices whose visited bit this query has just set) to the
 // warp's log.  Returns the new length, or -1 once the log is full: the query then falls back to zeroing
 // the words of its whole range.
 __device__ __forceinline__ int log_ranks(uint32_t* log, int cap, int n_logged, const uint32_t* cand, int ns, int lane) {
     if (n_logged + ns > cap) return -1;
-    if (lane < ns) __stcg(log + n_logged + lane, cand[lane]);
-    if (lane + 32 < ns) __stcg(log + n_logged + lane + 32, cand[lane + 32]);
+    for (int i = lane; i < ns; i += 32) __stcg(log + n_logged + i, cand[i]);
     return n_logged + ns;
 }
 

@@ -99,7 +99,7 @@ typedef void (*frog_kernel_fn)(const FrogSearchArgs);
 
 namespace froghost {
 // frog_search_lean.cu: the trimmed kernel for 384- and 512-byte fp32 rows (null: shape not covered)
-frog_kernel_fn lean_kernel(int ef_s, int row_bytes, bool table, size_t* smem_per_warp, int* warps_per_cta);
+frog_kernel_fn lean_kernel(int ef_s, int budget, int row_bytes, bool table, size_t* smem_per_warp, int* warps_per_cta);
 void set_cuda_error(cudaError_t e);
 int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in, frog_params_t* out);
 bool make_row_tensor_map(const void* base, bool f16, int row_elems, size_t row_bytes, size_t n, CUtensorMap* out);

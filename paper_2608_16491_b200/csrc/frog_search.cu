@@ -63,7 +63,7 @@ struct WarpSmem {
 };
 
 __host__ __device__ inline size_t warp_smem_bytes(int pool_slots, int q_len, int hash_bits, bool bitmap) {
-    const size_t b = (size_t)STAGE_BYTES + (size_t)pool_slots * 8 + 64 * 4 + 32 + (size_t)q_len * 4 +
+    const size_t b = (size_t)STAGE_BYTES + (size_t)pool_slots * 8 + FROG_MAX_BUDGET * 4 + 32 + (size_t)q_len * 4 +
                      (bitmap ? 0 : ((size_t)4 << hash_bits));
     return (b + 127) & ~(size_t)127;
 }
@@ -140,7 +140,7 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
     S.stage = reinterpret_cast<float4*>(base);
     S.pool = reinterpret_cast<uint64_t*>(base + STAGE_BYTES);
     S.cand = reinterpret_cast<uint32_t*>(S.pool + POOL);
-    S.bar = reinterpret_cast<uint64_t*>(S.cand + 64);
+    S.bar = reinterpret_cast<uint64_t*>(S.cand + FROG_MAX_BUDGET);
     S.q = reinterpret_cast<float4*>(S.bar + 4);
     S.hash = reinterpret_cast<uint32_t*>(reinterpret_cast<float*>(S.q) + A.q_len);
     if (lane == 0) {
@@ -277,8 +277,8 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                 // admitted lane applies the visited check where it stands (it stays lazy: entries
                 // already evaluated still consume budget); survivors are compacted into S.cand.
                 const uint32_t* hot = A.enc + ((size_t)u * A.H + L_start) * A.m;
-                // a trace record is appended only while 66 words (header + 64 entries) remain
-                const bool rec_ok = (MODE == MODE_TRACE) && trace_ok && (trace_len + 66 <= (uint32_t)A.trace_cap - 1);
+                // a trace record is appended only while a full one (header + max(64, B) entries) fits
+                const bool rec_ok = (MODE == MODE_TRACE) && trace_ok && (trace_len + 2 + (uint32_t)max(64, A.B) <= (uint32_t)A.trace_cap - 1);
                 int cnt = 0, scanned = 0;
                 ns = 0;
                 if (MODE == MODE_EAGER) {
@@ -399,14 +399,10 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
                     }
                 }
                 if (BITMAP && n_logged >= 0) n_logged = log_ranks(bitmap + A.bitmap_words, A.log_cap, n_logged, S.cand, ns, lane);
-                // lines 14-17; a budget above 32 can leave up to 64 survivors: two batches, the pool
-                // after both is the same as after one merge of all of them
-                if (ns > 32) {
-                    EVAL(32, 0u);
-                    first = EVAL(ns - 32, 0u, 32);
-                } else {
-                    first = EVAL(ns, 0u);
-                }
+                // lines 14-17; a budget above 32 can leave up to B survivors: batches of 32, the pool
+                // after all of them is the same as after one merge of everything
+                first = EVAL(min(ns, 32), 0u);
+                for (int off = 32; off < ns; off += 32) first = EVAL(min(ns - off, 32), 0u, off);
             }
             if (BITMAP && A.slab_clean) {
                 // leave the slab all-zero: the words of the logged ranks, or of the whole range
@@ -574,10 +570,10 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
         // FROG_VISITED_BITMAP keeps the bitmap
         table = allow_table && P.visited == FROG_VISITED_AUTO && beam_width <= 128 &&
                 (bitmap_words_per_slot(ix) >= (size_t)TABLE_MIN_SLAB_WORDS || (P.debug_flags & 8));
-        kernel_fn lean = froghost::lean_kernel(beam_width, ix->info.d_pad * 4, table, &per_warp, &wpc);
+        kernel_fn lean = froghost::lean_kernel(beam_width, P.budget, ix->info.d_pad * 4, table, &per_warp, &wpc);
         if (!lean && table) {
             table = false;
-            lean = froghost::lean_kernel(beam_width, ix->info.d_pad * 4, false, &per_warp, &wpc);
+            lean = froghost::lean_kernel(beam_width, P.budget, ix->info.d_pad * 4, false, &per_warp, &wpc);
         }
         if (lean && wpc == WARPS_PER_CTA) {
             fn = lean;

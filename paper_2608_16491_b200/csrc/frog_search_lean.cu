@@ -14,7 +14,8 @@
 //     were measured slower;
 //   * a team's leader stores its row's squared distance to shared memory, every lane picks up
 //     "its" distance with one load (no shuffle/compare chain to route results to lanes);
-//   * up to 64 survivors of one expansion go through one gather loop;
+//   * all survivors of one expansion (up to B: 64, or 128 in the instantiations for large budgets)
+//     go through one gather loop;
 //   * everything in the expansion loop is inlined (no call, no argument shuffling), the row
 //     geometry and the shared-memory layout are compile-time constants;
 //   * on indexes of 4M objects and more the visited set is a 16 KB hash table per warp that stays
@@ -81,21 +82,21 @@ __device__ unsigned long long g_lean_prof[8];
 #define LEAN_T(i) do { } while (0)
 #endif
 
-template <int EPL, int ROWB>
+template <int EPL, int ROWB, int CAP>
 struct Lean {
     static constexpr int NSLOT = ROWB <= 384 ? FROG_LEAN_NSLOT_384 : FROG_LEAN_NSLOT_512;   // quads in the ring
     static constexpr int QUAD = 4 * ROWB;                       // bytes of one quad
     static constexpr int POOL = 32 * EPL;
     static constexpr int OFF_POOL = NSLOT * QUAD;
-    static constexpr int OFF_CAND = OFF_POOL + POOL * 8;        // 64 ranks + 3 of padding + 1 spare
-    static constexpr int OFF_D2 = OFF_CAND + 72 * 4;            // squared distances of the <= 64 rows
-    static constexpr int OFF_Q = OFF_D2 + 64 * 4;               // query vector, ROWB bytes
+    static constexpr int OFF_CAND = OFF_POOL + POOL * 8;        // <= CAP (64 or 128) ranks + 3 of padding (+ 5 spare)
+    static constexpr int OFF_D2 = OFF_CAND + (CAP + 8) * 4;     // squared distances of the <= CAP rows
+    static constexpr int OFF_Q = OFF_D2 + CAP * 4;              // query vector, ROWB bytes
     static constexpr int OFF_BAR = OFF_Q + ROWB;                // NSLOT mbarriers, then the time-out flag
     static constexpr int BYTES = (OFF_BAR + 40 + 127) / 128 * 128;
     static_assert(OFF_CAND % 16 == 0 && OFF_Q % 16 == 0 && OFF_BAR % 8 == 0 && QUAD % 128 == 0, "alignment");
 };
 
-template <int EPL, int ROWB>
+template <int EPL, int ROWB, int CAP>
 struct LeanSmem {
     char* stage;
     uint64_t* pool;
@@ -105,7 +106,7 @@ struct LeanSmem {
     uint64_t* bar;
     uint32_t* timeout;
     __device__ __forceinline__ explicit LeanSmem(unsigned char* base) {
-        using L = Lean<EPL, ROWB>;
+        using L = Lean<EPL, ROWB, CAP>;
         stage = reinterpret_cast<char*>(base);
         pool = reinterpret_cast<uint64_t*>(base + L::OFF_POOL);
         cand = reinterpret_cast<uint32_t*>(base + L::OFF_CAND);
@@ -116,14 +117,14 @@ struct LeanSmem {
     }
 };
 
-// Squared distances of the ns <= 64 ranks in cand[0..ns) into d2[0..ns) (Alg. 2 line 14).  `ph`
+// Squared distances of the ns <= 128 ranks in cand[0..ns) into d2[0..ns) (Alg. 2 line 14).  `ph`
 // holds the parities of the ring's mbarriers.  Arithmetic order: lane s of an 8-lane team takes
 // the 4-float groups s, s+8, s+16, ... of its row in increasing order with fused multiply-adds,
 // then the partial sums are combined by a butterfly with partner distance 4, 2, 1.
-template <int EPL, int ROWB>
-__device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanSmem<EPL, ROWB>& S, int ns,
+template <int EPL, int ROWB, int CAP>
+__device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanSmem<EPL, ROWB, CAP>& S, int ns,
                                             uint32_t& ph, int lane) {
-    using L = Lean<EPL, ROWB>;
+    using L = Lean<EPL, ROWB, CAP>;
     const int groups = (ns + 3) >> 2;
     if (lane < 3) S.cand[ns + lane] = (uint32_t)A.n + 1u + (uint32_t)lane;    // rows beyond the tensor: zeros
     __syncwarp();
@@ -169,9 +170,10 @@ __device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanS
     __syncwarp();
 }
 
-// MergeTopEfS of the ns <= 64 evaluated candidates (lines 15-17); returns the first unexpanded position.
-template <int EPL, int ROWB>
-__device__ __forceinline__ int lean_merge(const LeanSmem<EPL, ROWB>& S, int ns, int ef_s, uint32_t new_flag, int off, int lane) {
+// MergeTopEfS of 32 of the ns <= 128 evaluated candidates, those from `off` on (lines 15-17: merging
+// them batch by batch leaves the pool that one merge of all would); returns the first unexpanded position.
+template <int EPL, int ROWB, int CAP>
+__device__ __forceinline__ int lean_merge(const LeanSmem<EPL, ROWB, CAP>& S, int ns, int ef_s, uint32_t new_flag, int off, int lane) {
     const int j = off + lane;
     const uint64_t key = (j < ns) ? make_key(S.d2[j], S.cand[j], new_flag) : KEY_EMPTY;
     return (int)merge_batch<EPL, true>(S.pool, key, ef_s, lane);
@@ -179,23 +181,23 @@ __device__ __forceinline__ int lean_merge(const LeanSmem<EPL, ROWB>& S, int ns, 
 
 // gather + merge out of line, for the places that run once per query (entry points, exact scan) and
 // the rare second batch of an expansion; returns first | parities << 16
-template <int EPL, int ROWB>
+template <int EPL, int ROWB, int CAP>
 __device__ __noinline__ uint32_t lean_eval_cold(const FrogSearchArgs& A, unsigned char* base, int ns, uint32_t new_flag,
                                                 uint32_t ph) {
-    const LeanSmem<EPL, ROWB> S(base);
+    const LeanSmem<EPL, ROWB, CAP> S(base);
     const int lane = lane_id();
-    lean_gather<EPL, ROWB>(A, S, ns, ph, lane);
-    int first = lean_merge<EPL, ROWB>(S, ns, A.ef_s, new_flag, 0, lane);
-    if (ns > 32) first = lean_merge<EPL, ROWB>(S, ns, A.ef_s, new_flag, 32, lane);
+    lean_gather<EPL, ROWB, CAP>(A, S, ns, ph, lane);
+    int first = lean_merge<EPL, ROWB, CAP>(S, ns, A.ef_s, new_flag, 0, lane);
+    for (int off = 32; off < ns; off += 32) first = lean_merge<EPL, ROWB, CAP>(S, ns, A.ef_s, new_flag, off, lane);
     return (uint32_t)first | (ph << 16);
 }
-template <int EPL, int ROWB>
+template <int EPL, int ROWB, int CAP>
 __device__ __noinline__ int lean_merge_cold(unsigned char* base, int ns, int ef_s, uint32_t new_flag, int off) {
-    const LeanSmem<EPL, ROWB> S(base);
-    return lean_merge<EPL, ROWB>(S, ns, ef_s, new_flag, off, lane_id());
+    const LeanSmem<EPL, ROWB, CAP> S(base);
+    return lean_merge<EPL, ROWB, CAP>(S, ns, ef_s, new_flag, off, lane_id());
 }
 
-// Visited check of the cnt <= 64 ranks in en[] (EN order): survivors are compacted, in order, into
+// Visited check of the cnt <= 64 ranks in en[] (EN order; a longer list is passed in two parts): survivors are compacted, in order, into
 // cand[]; returns their number.  Lane l looks after en[l] and en[l + 32].  With `table` the set is the
 // warp's hash table (L2-resident), otherwise its bitmap slab.
 __device__ __forceinline__ int lean_visit_list(const uint32_t* en, int cnt, uint32_t* cand, uint32_t* table, int table_bits,
@@ -227,15 +229,15 @@ __device__ __forceinline__ int lean_visit_list(const uint32_t* en, int cnt, uint
 // candidate costs no DRAM access; the bitmap's scattered read-modify-writes are what keeps DRAM from the
 // row gathers on large indexes).  The table is exact; a query that fills it half way moves its entries
 // to the warp's bitmap slab and carries on there.
-template <int EPL, int ROWB, bool TABLE>
+template <int EPL, int ROWB, bool TABLE, int CAP = 64>
 __global__ void __launch_bounds__(LEAN_WARPS * 32, lean_min_ctas(EPL, ROWB))
 frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
-    using L = Lean<EPL, ROWB>;
+    using L = Lean<EPL, ROWB, CAP>;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int lane = lane_id();
     const int warp = threadIdx.x >> 5;
     unsigned char* base = smem_raw + L::BYTES * warp;
-    const LeanSmem<EPL, ROWB> S(base);
+    const LeanSmem<EPL, ROWB, CAP> S(base);
     if (lane == 0) {
 #pragma unroll
         for (int i = 0; i < L::NSLOT; ++i) mbar_init(S.bar + i, 1u);
@@ -294,7 +296,7 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
                 if (lane < cnt) S.cand[lane] = (uint32_t)(l_q + b0 + lane);
                 if (lane + 32 < cnt) S.cand[lane + 32] = (uint32_t)(l_q + b0 + lane + 32);
                 __syncwarp();
-                ph = lean_eval_cold<EPL, ROWB>(A, base, cnt, 1u, ph) >> 16;
+                ph = lean_eval_cold<EPL, ROWB, CAP>(A, base, cnt, 1u, ph) >> 16;
                 __syncwarp();
             }
         } else {
@@ -338,7 +340,7 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
             if (n_logged >= 0) n_logged = log_ranks(bitmap + A.bitmap_words, A.log_cap, n_logged, S.cand, ns, lane);
             int first;
             {
-                const uint32_t r = lean_eval_cold<EPL, ROWB>(A, base, ns, 0u, ph);
+                const uint32_t r = lean_eval_cold<EPL, ROWB, CAP>(A, base, ns, 0u, ph);
                 first = (int)(r & 0xFFFFu);
                 ph = r >> 16;
             }
@@ -350,7 +352,7 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
                 const uint32_t u = key_rank(S.pool[first]);               // line 8
                 __syncwarp();
                 if (lane == 0) S.pool[first] |= 1ull;                     // line 9
-                if (TABLE && table && n_seen + 64 > (1 << (A.table_bits - 1))) {
+                if (TABLE && table && n_seen + A.B > (1 << (A.table_bits - 1))) {
                     // the next expansion could take the table past half full: move every rank to the
                     // bitmap slab (all-zero until now) and carry on there; the slab is zeroed by range at the end
                     for (int i = lane; i < (1 << A.table_bits); i += 32) {
@@ -427,17 +429,20 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
                 }
                 __syncwarp();
                 if (TABLE) {
-                    ns = lean_visit_list(en, cnt, S.cand, table, A.table_bits, bitmap, keep_in_l2, S.timeout, lane);
+                    ns = lean_visit_list(en, min(cnt, 64), S.cand, table, A.table_bits, bitmap, keep_in_l2, S.timeout, lane);
+                    if (cnt > 64)
+                        ns += lean_visit_list(en + 64, cnt - 64, S.cand + ns, table, A.table_bits, bitmap, keep_in_l2,
+                                              S.timeout, lane);
                     n_seen += ns;
                 }
                 ++n_exp;
                 if (n_logged >= 0) n_logged = log_ranks(bitmap + A.bitmap_words, A.log_cap, n_logged, S.cand, ns, lane);
                 // lines 14-17
                 LEAN_T(1);
-                lean_gather<EPL, ROWB>(A, S, ns, ph, lane);
+                lean_gather<EPL, ROWB, CAP>(A, S, ns, ph, lane);
                 LEAN_T(2);
-                first = lean_merge<EPL, ROWB>(S, ns, A.ef_s, 0u, 0, lane);
-                if (ns > 32) first = lean_merge_cold<EPL, ROWB>(base, ns, A.ef_s, 0u, 32);
+                first = lean_merge<EPL, ROWB, CAP>(S, ns, A.ef_s, 0u, 0, lane);
+                for (int off = 32; off < ns; off += 32) first = lean_merge_cold<EPL, ROWB, CAP>(base, ns, A.ef_s, 0u, off);
                 LEAN_T(3);
 #ifdef FROG_LEAN_PROFILE
                 t_ph[6] += 1;
@@ -497,15 +502,26 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
 #endif
 }
 
+// Budgets up to 64 get the compact shared-memory layout (CAP = 64: what keeps 32-36 warps resident
+// inside the 196 KB carve-out, so that L1 keeps 60 KB; the larger layout was measured 4-9 % slower at
+// B <= 64); budgets up to 128 are instantiated for the pools of 128-256 keys, where they pay (hard,
+// narrow-range batches); other combinations go to the general kernel.
 template <int ROWB>
-frog_kernel_fn lean_pick(int ef_s, bool table, size_t* smem_per_warp) {
-    if (ef_s <= 32) { *smem_per_warp = Lean<1, ROWB>::BYTES; return table ? frog_search_lean_kernel<1, ROWB, true> : frog_search_lean_kernel<1, ROWB, false>; }
-    if (ef_s <= 64) { *smem_per_warp = Lean<2, ROWB>::BYTES; return table ? frog_search_lean_kernel<2, ROWB, true> : frog_search_lean_kernel<2, ROWB, false>; }
-    if (ef_s <= 128) { *smem_per_warp = Lean<4, ROWB>::BYTES; return table ? frog_search_lean_kernel<4, ROWB, true> : frog_search_lean_kernel<4, ROWB, false>; }
+frog_kernel_fn lean_pick(int ef_s, int budget, bool table, size_t* smem_per_warp) {
+    if (budget > 64) {
+        if (ef_s <= 64 || ef_s > 256 || (table && ef_s > 128)) return nullptr;
+        if (ef_s <= 128) { *smem_per_warp = Lean<4, ROWB, 128>::BYTES; return table ? frog_search_lean_kernel<4, ROWB, true, 128> : frog_search_lean_kernel<4, ROWB, false, 128>; }
+        if (ef_s <= 192) { *smem_per_warp = Lean<6, ROWB, 128>::BYTES; return frog_search_lean_kernel<6, ROWB, false, 128>; }
+        *smem_per_warp = Lean<8, ROWB, 128>::BYTES;
+        return frog_search_lean_kernel<8, ROWB, false, 128>;
+    }
+    if (ef_s <= 32) { *smem_per_warp = Lean<1, ROWB, 64>::BYTES; return table ? frog_search_lean_kernel<1, ROWB, true> : frog_search_lean_kernel<1, ROWB, false>; }
+    if (ef_s <= 64) { *smem_per_warp = Lean<2, ROWB, 64>::BYTES; return table ? frog_search_lean_kernel<2, ROWB, true> : frog_search_lean_kernel<2, ROWB, false>; }
+    if (ef_s <= 128) { *smem_per_warp = Lean<4, ROWB, 64>::BYTES; return table ? frog_search_lean_kernel<4, ROWB, true> : frog_search_lean_kernel<4, ROWB, false>; }
     if (table) return nullptr;
-    if (ef_s <= 192) { *smem_per_warp = Lean<6, ROWB>::BYTES; return frog_search_lean_kernel<6, ROWB, false>; }
-    if (ef_s <= 256) { *smem_per_warp = Lean<8, ROWB>::BYTES; return frog_search_lean_kernel<8, ROWB, false>; }
-    *smem_per_warp = Lean<16, ROWB>::BYTES;
+    if (ef_s <= 192) { *smem_per_warp = Lean<6, ROWB, 64>::BYTES; return frog_search_lean_kernel<6, ROWB, false>; }
+    if (ef_s <= 256) { *smem_per_warp = Lean<8, ROWB, 64>::BYTES; return frog_search_lean_kernel<8, ROWB, false>; }
+    *smem_per_warp = Lean<16, ROWB, 64>::BYTES;
     return frog_search_lean_kernel<16, ROWB, false>;
 }
 
@@ -516,10 +532,10 @@ namespace froghost {
 // The lean kernel for this beam width and row size, or null if the shape is not covered (the caller
 // then uses the generic kernel).  Needs the row tensor map and the bitmap visited set.  `table`: the
 // variant whose visited set is the L2-resident hash table (pools of up to 128 keys only).
-frog_kernel_fn lean_kernel(int ef_s, int row_bytes, bool table, size_t* smem_per_warp, int* warps_per_cta) {
+frog_kernel_fn lean_kernel(int ef_s, int budget, int row_bytes, bool table, size_t* smem_per_warp, int* warps_per_cta) {
     *warps_per_cta = LEAN_WARPS;
-    if (row_bytes == 384) return lean_pick<384>(ef_s, table, smem_per_warp);
-    if (row_bytes == 512) return lean_pick<512>(ef_s, table, smem_per_warp);
+    if (row_bytes == 384) return lean_pick<384>(ef_s, budget, table, smem_per_warp);
+    if (row_bytes == 512) return lean_pick<512>(ef_s, budget, table, smem_per_warp);
     return nullptr;
 }
 

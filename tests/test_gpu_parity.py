@@ -246,7 +246,7 @@ def test_empty_batch_and_argument_errors(libs, tiny_gpu):
     with pytest.raises(libs.FrogError):
         gix.search(q, lo, hi, 10, 32, params=libs.Params(epn=33))
     with pytest.raises(libs.FrogError):
-        gix.search(q, lo, hi, 10, 32, params=libs.Params(budget=65))
+        gix.search(q, lo, hi, 10, 32, params=libs.Params(budget=129))
     with pytest.raises(libs.FrogError):
         gix.search(q, lo, hi, 10, 32, params=libs.Params(exact_below=-1))
     with pytest.raises(libs.FrogError):                  # the ablation exists for the bitmap form only
@@ -310,7 +310,8 @@ def test_scaled_workloads_match_oracle(libs, cache_dir, name, n, nq):
     try:
         for ef, k, B, vis in ((32, 10, 16, libs.VISITED_BITMAP), (100, 100, 16, libs.VISITED_HASH),
                               (64, 10, 32, libs.VISITED_BITMAP), (48, 10, 24, libs.VISITED_HASH),
-                              (48, 10, 64, libs.VISITED_BITMAP)):
+                              (48, 10, 64, libs.VISITED_BITMAP), (32, 10, 96, libs.VISITED_BITMAP),
+                              (40, 10, 128, libs.VISITED_HASH), (24, 10, 128, libs.VISITED_BITMAP)):
             ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef, B=B, trace_cap=60000)
             got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, k, ef, trace_cap=60000, budget=B, visited=vis)
             _assert_parity(got, ref, slots=_default_slots(ef))
@@ -334,7 +335,8 @@ def test_row_specialised_kernel_at_every_pool_size(libs, cache_dir, name, n, nq)
     gix = libs.Index.load(path, 0)
     try:
         for ef, k, kw in ((24, 10, dict(budget=64)), (64, 64, dict(budget=64, epn=32)), (128, 10, dict(budget=64)),
-                          (176, 10, dict(budget=64)), (200, 100, dict(budget=48)), (256, 10, dict(budget=64, max_iters=40)),
+                          (176, 10, dict(budget=64)), (32, 10, dict(budget=96)), (160, 10, dict(budget=128)),
+                          (200, 100, dict(budget=48)), (256, 10, dict(budget=64, max_iters=40)),
                           (512, 10, dict(budget=64)), (96, 10, dict(budget=64, exact_below=2000)),
                           (40, 10, dict(budget=64, no_hotspot=1, seed=9))):
             ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef, epn=kw.get("epn", 16), B=kw["budget"],
@@ -361,7 +363,7 @@ def test_visited_hash_table_form(libs, cache_dir, name, n, nq):
     gix = libs.Index.load(path, 0)
     try:
         q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
-        for ef, k, B in ((32, 10, 64), (64, 10, 64), (24, 5, 16), (48, 48, 33)):
+        for ef, k, B in ((32, 10, 64), (64, 10, 64), (24, 5, 16), (48, 48, 33), (24, 10, 96), (100, 10, 128)):
             ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef, B=B)
             for bits in (0, 8, 6, 0):
                 prm = libs.Params(budget=B, debug_flags=8 | (bits << 8))
