@@ -40,7 +40,7 @@ if ROOT not in sys.path:
 METRIC = "mixed-selectivity QPS at recall@10>=0.95"
 UNIT = "queries/s"
 SWEEP = [16, 24, 32, 40, 44, 48, 52, 56, 64, 80, 96, 112, 128, 160, 192, 256, 320, 384, 448, 512]
-SECONDARY_BUDGETS = [32, 64, 96]  # ... for the entries of config.per_workload and the reference arm's choice
+SECONDARY_BUDGETS = [32, 64, 96, 128]  # ... for the entries of config.per_workload and the reference arm's choice
 BUDGETS = [16, 32, 48, 64, 96]  # expansion budget B of Alg. 2: from the paper's default upwards (the kernels take up to 128)
 RECALL_TARGET = 0.95
 HBM_FALLBACK_GBS = 6650.0

@@ -123,7 +123,7 @@ def _room_or_skip(name, n, d, m):
 
 
 @pytest.mark.parametrize("name,k,beam,BUDGET", [("deep1m", 10, 192, 64), ("deep1m", 10, 128, 32), ("deep1m", 10, 128, 96), ("text", 10, 512, 64),
-                                                ("text", 10, 320, 96), ("deep10m", 10, 32, 64), ("deep10m", 100, 128, 64)])
+                                                ("text", 10, 192, 128), ("deep10m", 10, 32, 64), ("deep10m", 100, 128, 64)])
 def test_other_workloads_at_full_size(libs, name, k, beam, BUDGET):
     if os.environ.get("FROG_SKIP_FULLSIZE") == "1":
         pytest.skip("FROG_SKIP_FULLSIZE=1")

@@ -311,7 +311,8 @@ def test_scaled_workloads_match_oracle(libs, cache_dir, name, n, nq):
         for ef, k, B, vis in ((32, 10, 16, libs.VISITED_BITMAP), (100, 100, 16, libs.VISITED_HASH),
                               (64, 10, 32, libs.VISITED_BITMAP), (48, 10, 24, libs.VISITED_HASH),
                               (48, 10, 64, libs.VISITED_BITMAP), (32, 10, 96, libs.VISITED_BITMAP),
-                              (40, 10, 128, libs.VISITED_HASH), (24, 10, 128, libs.VISITED_BITMAP)):
+                              (40, 10, 128, libs.VISITED_HASH), (24, 10, 128, libs.VISITED_BITMAP),
+                              (300, 10, 96, libs.VISITED_BITMAP)):
             ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, k, ef, B=B, trace_cap=60000)
             got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, k, ef, trace_cap=60000, budget=B, visited=vis)
             _assert_parity(got, ref, slots=_default_slots(ef))
