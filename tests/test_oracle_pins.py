@@ -159,7 +159,7 @@ def test_en_identification_is_order_preserving_prefix():
         r = int(rng.integers(l, 200))
         ls = int(rng.integers(0, H))
         le = int(rng.integers(ls, H))
-        B = int(rng.integers(1, 33))
+        B = int(rng.integers(1, 33)) if rng.random() < 0.5 else int(rng.integers(33, 200))   # up to and beyond the kernels' 128
         flat = enc[ls:le + 1].ravel()
         expect = [int(v) for v in flat if v != 0xFFFFFFFF and l <= v <= r][:B]
         got = None
