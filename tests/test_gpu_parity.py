@@ -162,7 +162,7 @@ def test_concurrent_streams_share_one_index(libs, tiny_gpu):
     separate calls.  More streams than scratch sets exist are served too (they queue)."""
     wl, ix, gix = tiny_gpu
     q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
-    cfgs = [(32, 64), (96, 16), (48, 32), (64, 64), (24, 8), (128, 16)]          # (beam, budget) per stream
+    cfgs = [(32, 64), (96, 16), (48, 32), (64, 64), (24, 8), (128, 16), (100, 128)]   # (beam, budget) per stream
     refs = [oracle.search(ix, wl.queries, wl.lo, wl.hi, wl.k, ef, B=B) for ef, B in cfgs]
     streams = [torch.cuda.Stream() for _ in cfgs]
     torch.cuda.synchronize()
