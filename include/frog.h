@@ -75,6 +75,13 @@ typedef struct {
                                   (same results; for comparing the two);
                            bit 3: use the visited hash table (see FROG_VISITED_AUTO) on small indexes too;
                            bit 4: record CUDA events around the search kernel alone (frog_search_kernel_ms);
+                           bit 5: test of the error path: the kernel requests no row copy and its (bounded)
+                                  waits give up after 64 polls, so every gather ends as a copy time-out would,
+                                  with nothing in flight: the affected rows are padding, their status carries
+                                  FROG_ST_COPY_TIMEOUT, frog_search_last_status reports it, and the next call
+                                  works.  Honoured by the kernel for 384- and 512-byte rows (bitmap visited set,
+                                  beam widths up to 32, budgets up to 64) and, when `stats` is given, by the
+                                  general kernel; ignored otherwise;
                            bits 8-11: log2 of that table's slots, 6..12 (0 = 12), to make queries outgrow it */
     int32_t exact_below;/* ranges holding at most max(beam_width, exact_below) objects are answered by
                            scanning their contiguous rank slab (exact, status FROG_ST_EXACT) instead of

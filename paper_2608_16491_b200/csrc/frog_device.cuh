@@ -381,12 +381,14 @@ __device__ __forceinline__ float staged_dist2(const float* __restrict__ vectors,
 // group is up to 8 rows (4 for 512-byte slots: one row per team); a row longer than STAGE_CHUNK is
 // taken in column chunks, one chunk of every row of the group per step.  bar[0], bar[1] are the
 // two mbarriers; `phases` holds their parities in bits 0 and 1.
-template <bool F16, int ROWB = 0>
+// HOOKABLE && hook (tests of the error path): no copy is armed or issued and a wait gives up after 64
+// polls, so the routine reports a time-out with nothing in flight.
+template <bool F16, int ROWB = 0, bool HOOKABLE = false>
 __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows, int row_bytes, int slot_bytes,
                                                    const float4* qs, float4* stage, uint64_t* bar,
                                                    uint32_t& phases, bool& ok, uint32_t my_rank, int ns, int lane,
                                                    const void* tmap = nullptr, const uint32_t* ranks = nullptr,
-                                                   int n_rows_total = 0) {
+                                                   int n_rows_total = 0, bool hook = false) {
     if (ROWB > 0) {
         row_bytes = ROWB;
         slot_bytes = ROWB >= STAGE_CHUNK ? STAGE_CHUNK : ROWB;
@@ -409,7 +411,9 @@ __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows
         const int r0 = ig * rph, nrows = min(rph, ns - r0);
         const int c0 = ic * STAGE_CHUNK, cbytes = min(STAGE_CHUNK, row_bytes - c0);
         uint64_t* b = bar + (s & 1);
-        if (tmap) {
+        if (HOOKABLE && hook) {
+            // nothing is requested
+        } else if (tmap) {
             if (lane == 0) {
                 const int quads = (nrows + 3) >> 2;
                 mbar_expect_tx(b, (uint32_t)(quads * 4 * box_bytes));
@@ -443,7 +447,7 @@ __device__ __forceinline__ float staged_dist2_pipe(const void* __restrict__ rows
 #pragma unroll 1
     for (int s = 0; s < steps; ++s) {
         const int h = s & 1;
-        ok = mbar_wait(bar + h, (phases >> h) & 1u) && ok;
+        ok = ((HOOKABLE && hook) ? mbar_wait_limit(bar + h, (phases >> h) & 1u, 64) : mbar_wait(bar + h, (phases >> h) & 1u)) && ok;
         phases ^= 1u << h;
         const int r0 = g * rph, nrows = min(rph, ns - r0);
         const int c0 = c * STAGE_CHUNK, cbytes = min(STAGE_CHUNK, row_bytes - c0);

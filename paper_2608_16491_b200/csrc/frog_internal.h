@@ -92,6 +92,8 @@ struct FrogSearchArgs {
     int slot_bytes;            // bytes of one row slot in the stage buffer (multiple of 16, <= 512)
     int q_len;                 // floats of the query held in shared memory (8 * ceil(d / 8))
     int gather4;               // nonzero: `tmap` is valid and rows are fetched four per copy instruction
+    int no_copies;             // test hook of the counting variant: no row copy is armed or issued, waits give up
+                               // after 64 polls (every gather takes the time-out branch, nothing is in flight)
     alignas(64) CUtensorMap tmap;
 };
 
@@ -99,7 +101,8 @@ typedef void (*frog_kernel_fn)(const FrogSearchArgs);
 
 namespace froghost {
 // frog_search_lean.cu: the trimmed kernel for 384- and 512-byte fp32 rows (null: shape not covered)
-frog_kernel_fn lean_kernel(int ef_s, int budget, int row_bytes, bool table, size_t* smem_per_warp, int* warps_per_cta);
+frog_kernel_fn lean_kernel(int ef_s, int budget, int row_bytes, bool table, bool hook, size_t* smem_per_warp,
+                           int* warps_per_cta);
 void set_cuda_error(cudaError_t e);
 int resolve_params(const frog_index* ix, int beam_width, const frog_params_t* in, frog_params_t* out);
 bool make_row_tensor_map(const void* base, bool f16, int row_elems, size_t row_bytes, size_t n, CUtensorMap* out);

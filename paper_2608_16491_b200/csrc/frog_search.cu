@@ -85,11 +85,11 @@ __device__ __forceinline__ bool visited_test_and_set(const WarpSmem& S, uint32_t
 // lines 14-17).  Returns the first unexpanded pool position.  Kept out of line: it is called from
 // several places of the kernel and inlining every copy costs registers and instruction cache.
 // UNIQUE: the visited set is exact (bitmap form), so the ranks are distinct and none is in the pool.
-template <int EPL, bool F16, int ROWB, bool UNIQUE>
+template <int EPL, bool F16, int ROWB, bool UNIQUE, bool HOOKABLE = false>
 __device__ __noinline__ int evaluate_and_merge(const void* __restrict__ rows, int row_bytes, int slot_bytes, int ef_s,
                                                uint64_t* pool, const uint32_t* cand, uint64_t* bar,
                                                const float4* qs, float4* stage, int ns, uint32_t new_flag,
-                                               const void* tmap, int n, long long* t_dist) {
+                                               const void* tmap, int n, long long* t_dist, bool hook = false) {
     const int lane = lane_id();
     uint32_t id = (lane < ns) ? cand[lane] : 0u;
     if (!UNIQUE) {
@@ -112,8 +112,8 @@ __device__ __noinline__ int evaluate_and_merge(const void* __restrict__ rows, in
         __syncwarp();                       // lane 0's update of the parity in the previous call
         uint32_t phase = bar_words[0];
         bool ok = true;
-        d2 = staged_dist2_pipe<F16, ROWB>(rows, row_bytes, slot_bytes, qs, stage, bar, phase, ok, id, ns, lane,
-                                          UNIQUE ? tmap : nullptr, cand, n);
+        d2 = staged_dist2_pipe<F16, ROWB, HOOKABLE>(rows, row_bytes, slot_bytes, qs, stage, bar, phase, ok, id, ns, lane,
+                                                    UNIQUE ? tmap : nullptr, cand, n, hook);
         __syncwarp();                       // every lane has read the old parity
         if (lane == 0) {
             bar_words[0] = phase;
@@ -177,10 +177,10 @@ frog_search_kernel(const __grid_constant__ FrogSearchArgs A) {
         // distance + merge call; in profile builds the time is split at the end of the distances
         long long t_split = 0;
         auto EVAL = [&](int ns_, uint32_t flag_, int off_ = 0) {
-            int f_ = evaluate_and_merge<EPL, F16, ROWB, BITMAP>(A.rows, A.row_bytes, A.slot_bytes, A.ef_s, S.pool,
-                                                  S.cand + off_, S.bar, S.q, S.stage, ns_, flag_,
-                                                  A.gather4 ? &A.tmap : nullptr, A.n,
-                                                  MODE == MODE_PROFILE ? &t_split : nullptr);
+            int f_ = evaluate_and_merge<EPL, F16, ROWB, BITMAP, MODE == MODE_COUNT>(
+                A.rows, A.row_bytes, A.slot_bytes, A.ef_s, S.pool, S.cand + off_, S.bar, S.q, S.stage, ns_, flag_,
+                A.gather4 ? &A.tmap : nullptr, A.n, MODE == MODE_PROFILE ? &t_split : nullptr,
+                MODE == MODE_COUNT && A.no_copies != 0);
             if (MODE == MODE_PROFILE) {
                 long long n_ = clock64();
                 t_ph[3] += t_split - t_mark;
@@ -568,12 +568,13 @@ int plan_launch(const frog_index* ix, int beam_width, const frog_params_t& P, in
         // 4,194,304 objects and more: measured 1.26x faster at 10M objects, 0.85x at 1M, where the bits a
         // query touches still fit L2) and the pool is small enough for a query to fit the table as a rule;
         // FROG_VISITED_BITMAP keeps the bitmap
-        table = allow_table && P.visited == FROG_VISITED_AUTO && beam_width <= 128 &&
+        const bool hook = (P.debug_flags & 32) != 0;
+        table = allow_table && !hook && P.visited == FROG_VISITED_AUTO && beam_width <= 128 &&
                 (bitmap_words_per_slot(ix) >= (size_t)TABLE_MIN_SLAB_WORDS || (P.debug_flags & 8));
-        kernel_fn lean = froghost::lean_kernel(beam_width, P.budget, ix->info.d_pad * 4, table, &per_warp, &wpc);
+        kernel_fn lean = froghost::lean_kernel(beam_width, P.budget, ix->info.d_pad * 4, table, hook, &per_warp, &wpc);
         if (!lean && table) {
             table = false;
-            lean = froghost::lean_kernel(beam_width, P.budget, ix->info.d_pad * 4, false, &per_warp, &wpc);
+            lean = froghost::lean_kernel(beam_width, P.budget, ix->info.d_pad * 4, false, hook, &per_warp, &wpc);
         }
         if (lean && wpc == WARPS_PER_CTA) {
             fn = lean;
@@ -608,6 +609,7 @@ void set_gather(const frog_index* ix, bool f16, FrogSearchArgs* A) {
     A->row_bytes = f16 ? d_pad_h * 2 : ix->info.d_pad * 4;
     A->slot_bytes = A->row_bytes < STAGE_CHUNK ? A->row_bytes : STAGE_CHUNK;   // rows are 16-byte multiples
     A->q_len = d_pad_h;
+    A->no_copies = 0;
     A->gather4 = FROG_GATHER4 && (f16 ? ix->has_tmap_f16 : ix->has_tmap_f32);
     if (A->gather4) A->tmap = f16 ? ix->tmap_f16 : ix->tmap_f32;
     else std::memset(&A->tmap, 0, sizeof(A->tmap));
@@ -899,6 +901,7 @@ extern "C" int frog_search_ex(const frog_index_t* index, const float* queries, c
     A.ranges = nullptr;
     A.order = nullptr;
     set_gather(index, P.storage == FROG_STORAGE_F16, &A);
+    A.no_copies = (P.debug_flags & 32) ? 1 : 0;             // tests of the error path (see frog.h)
 
     FROG_CUDA_TRY(cudaMemsetAsync(sc->d_work, 0, 1024, s));
     // planning pass (skipped for tiny batches and when its scratch cannot be had)

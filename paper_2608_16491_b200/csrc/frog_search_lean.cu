@@ -121,7 +121,9 @@ struct LeanSmem {
 // holds the parities of the ring's mbarriers.  Arithmetic order: lane s of an 8-lane team takes
 // the 4-float groups s, s+8, s+16, ... of its row in increasing order with fused multiply-adds,
 // then the partial sums are combined by a butterfly with partner distance 4, 2, 1.
-template <int EPL, int ROWB, int CAP>
+// HOOK (an instantiation of its own, for the test of the error path): no copy is armed or issued and a
+// wait gives up after 64 polls, so every gather ends in the time-out branch without anything in flight.
+template <int EPL, int ROWB, int CAP, bool HOOK = false>
 __device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanSmem<EPL, ROWB, CAP>& S, int ns,
                                             uint32_t& ph, int lane) {
     using L = Lean<EPL, ROWB, CAP>;
@@ -130,6 +132,7 @@ __device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanS
     __syncwarp();
     const uint64_t policy = l2_policy_evict_first();                           // rows are read about once per batch
     auto issue = [&](int g, int slot) {
+        if (HOOK) return;
         uint64_t* b = S.bar + slot;
         mbar_expect_tx(b, (uint32_t)L::QUAD);
         const uint4 rk = *reinterpret_cast<const uint4*>(S.cand + 4 * g);
@@ -145,7 +148,7 @@ __device__ __forceinline__ void lean_gather(const FrogSearchArgs& A, const LeanS
     int slot = 0;
 #pragma unroll 1
     for (int g = 0; g < groups; ++g) {
-        if (!mbar_wait(S.bar + slot, (ph >> slot) & 1u)) *S.timeout = 1u;
+        if (!(HOOK ? mbar_wait_limit(S.bar + slot, (ph >> slot) & 1u, 64) : mbar_wait(S.bar + slot, (ph >> slot) & 1u))) *S.timeout = 1u;
         ph ^= 1u << slot;
         const char* x = mine + slot * L::QUAD;
         float a = 0.f;
@@ -181,12 +184,12 @@ __device__ __forceinline__ int lean_merge(const LeanSmem<EPL, ROWB, CAP>& S, int
 
 // gather + merge out of line, for the places that run once per query (entry points, exact scan) and
 // the rare second batch of an expansion; returns first | parities << 16
-template <int EPL, int ROWB, int CAP>
+template <int EPL, int ROWB, int CAP, bool HOOK = false>
 __device__ __noinline__ uint32_t lean_eval_cold(const FrogSearchArgs& A, unsigned char* base, int ns, uint32_t new_flag,
                                                 uint32_t ph) {
     const LeanSmem<EPL, ROWB, CAP> S(base);
     const int lane = lane_id();
-    lean_gather<EPL, ROWB, CAP>(A, S, ns, ph, lane);
+    lean_gather<EPL, ROWB, CAP, HOOK>(A, S, ns, ph, lane);
     int first = lean_merge<EPL, ROWB, CAP>(S, ns, A.ef_s, new_flag, 0, lane);
     for (int off = 32; off < ns; off += 32) first = lean_merge<EPL, ROWB, CAP>(S, ns, A.ef_s, new_flag, off, lane);
     return (uint32_t)first | (ph << 16);
@@ -229,7 +232,7 @@ __device__ __forceinline__ int lean_visit_list(const uint32_t* en, int cnt, uint
 // candidate costs no DRAM access; the bitmap's scattered read-modify-writes are what keeps DRAM from the
 // row gathers on large indexes).  The table is exact; a query that fills it half way moves its entries
 // to the warp's bitmap slab and carries on there.
-template <int EPL, int ROWB, bool TABLE, int CAP = 64>
+template <int EPL, int ROWB, bool TABLE, int CAP = 64, bool HOOK = false>
 __global__ void __launch_bounds__(LEAN_WARPS * 32, lean_min_ctas(EPL, ROWB))
 frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
     using L = Lean<EPL, ROWB, CAP>;
@@ -296,7 +299,7 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
                 if (lane < cnt) S.cand[lane] = (uint32_t)(l_q + b0 + lane);
                 if (lane + 32 < cnt) S.cand[lane + 32] = (uint32_t)(l_q + b0 + lane + 32);
                 __syncwarp();
-                ph = lean_eval_cold<EPL, ROWB, CAP>(A, base, cnt, 1u, ph) >> 16;
+                ph = lean_eval_cold<EPL, ROWB, CAP, HOOK>(A, base, cnt, 1u, ph) >> 16;
                 __syncwarp();
             }
         } else {
@@ -340,7 +343,7 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
             if (n_logged >= 0) n_logged = log_ranks(bitmap + A.bitmap_words, A.log_cap, n_logged, S.cand, ns, lane);
             int first;
             {
-                const uint32_t r = lean_eval_cold<EPL, ROWB, CAP>(A, base, ns, 0u, ph);
+                const uint32_t r = lean_eval_cold<EPL, ROWB, CAP, HOOK>(A, base, ns, 0u, ph);
                 first = (int)(r & 0xFFFFu);
                 ph = r >> 16;
             }
@@ -439,7 +442,7 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
                 if (n_logged >= 0) n_logged = log_ranks(bitmap + A.bitmap_words, A.log_cap, n_logged, S.cand, ns, lane);
                 // lines 14-17
                 LEAN_T(1);
-                lean_gather<EPL, ROWB, CAP>(A, S, ns, ph, lane);
+                lean_gather<EPL, ROWB, CAP, HOOK>(A, S, ns, ph, lane);
                 LEAN_T(2);
                 first = lean_merge<EPL, ROWB, CAP>(S, ns, A.ef_s, 0u, 0, lane);
                 for (int off = 32; off < ns; off += 32) first = lean_merge_cold<EPL, ROWB, CAP>(base, ns, A.ef_s, 0u, off);
@@ -507,7 +510,12 @@ frog_search_lean_kernel(const __grid_constant__ FrogSearchArgs A) {
 // B <= 64); budgets up to 128 are instantiated for the pools of 128-256 keys, where they pay (hard,
 // narrow-range batches); other combinations go to the general kernel.
 template <int ROWB>
-frog_kernel_fn lean_pick(int ef_s, int budget, bool table, size_t* smem_per_warp) {
+frog_kernel_fn lean_pick(int ef_s, int budget, bool table, bool hook, size_t* smem_per_warp) {
+    if (hook) {
+        if (table || budget > 64 || ef_s > 32) return nullptr;
+        *smem_per_warp = Lean<1, ROWB, 64>::BYTES;
+        return frog_search_lean_kernel<1, ROWB, false, 64, true>;
+    }
     if (budget > 64) {
         if (ef_s <= 64 || ef_s > 256 || (table && ef_s > 128)) return nullptr;
         if (ef_s <= 128) { *smem_per_warp = Lean<4, ROWB, 128>::BYTES; return table ? frog_search_lean_kernel<4, ROWB, true, 128> : frog_search_lean_kernel<4, ROWB, false, 128>; }
@@ -531,11 +539,13 @@ namespace froghost {
 
 // The lean kernel for this beam width and row size, or null if the shape is not covered (the caller
 // then uses the generic kernel).  Needs the row tensor map and the bitmap visited set.  `table`: the
-// variant whose visited set is the L2-resident hash table (pools of up to 128 keys only).
-frog_kernel_fn lean_kernel(int ef_s, int budget, int row_bytes, bool table, size_t* smem_per_warp, int* warps_per_cta) {
+// variant whose visited set is the L2-resident hash table (pools of up to 128 keys only); `hook`: the
+// instantiation whose gathers time out by construction (bitmap form, beams up to 32, budgets up to 64).
+frog_kernel_fn lean_kernel(int ef_s, int budget, int row_bytes, bool table, bool hook, size_t* smem_per_warp,
+                           int* warps_per_cta) {
     *warps_per_cta = LEAN_WARPS;
-    if (row_bytes == 384) return lean_pick<384>(ef_s, budget, table, smem_per_warp);
-    if (row_bytes == 512) return lean_pick<512>(ef_s, budget, table, smem_per_warp);
+    if (row_bytes == 384) return lean_pick<384>(ef_s, budget, table, hook, smem_per_warp);
+    if (row_bytes == 512) return lean_pick<512>(ef_s, budget, table, hook, smem_per_warp);
     return nullptr;
 }
 

@@ -353,6 +353,46 @@ def test_row_specialised_kernel_at_every_pool_size(libs, cache_dir, name, n, nq)
         gix.close()
 
 
+@pytest.mark.parametrize("name,n,nq", [("sift", 60_000, 300), ("deep1m", 50_000, 300), ("text", 20_000, 150)])
+def test_a_row_copy_that_never_completes_is_reported(libs, cache_dir, name, n, nq):
+    """The error path of the search kernels, exercised without a fault: with debug_flags bit 5 the kernel
+    requests no row copy and its bounded waits give up after 64 polls, so every gather ends the way a
+    copy time-out would, with nothing in flight.  Every row is then padding, every query that had
+    anything to evaluate carries FROG_ST_COPY_TIMEOUT, the launch-wide status word reports it to a
+    caller that passed no status array, and the next call on the same index answers normally.
+    Without `stats` the kernel for 384- and 512-byte rows runs (the general one for other rows, which
+    ignores the flag there: its plain form is checked through the counting variant), with `stats` the
+    counting variant of the general kernel."""
+    from conftest import build_scaled
+    wl, path, ix = build_scaled(libs, cache_dir, name, n, nq)
+    gix = libs.Index.load(path, 0)
+    try:
+        q, lo, hi = _dev(wl.queries), _dev(wl.lo), _dev(wl.hi)
+        ref = oracle.search(ix, wl.queries, wl.lo, wl.hi, 10, 32, B=64)
+        nonempty = (ref.status & 1) == 0
+        assert nonempty.sum() > nq // 2
+        prm = libs.Params(budget=64, debug_flags=32)
+        for with_stats in ([False, True] if name != "text" else [True]):
+            status = torch.zeros(nq, dtype=torch.int32, device="cuda")
+            stats = torch.zeros((nq, 4), dtype=torch.int32, device="cuda") if with_stats else None
+            ids, dists = gix.search(q, lo, hi, 10, 32, params=prm, status=status, stats=stats)
+            torch.cuda.synchronize()
+            st = status.cpu().numpy().view(np.uint32)
+            assert (ids.cpu().numpy() == -1).all() and np.isinf(dists.cpu().numpy()).all(), with_stats
+            assert ((st[nonempty] & 32) != 0).all(), with_stats
+            assert gix.last_status() & 32, with_stats
+            # the same launch for a caller without a status array: the launch-wide word still tells
+            gix.search(q, lo, hi, 10, 32, params=prm, stats=stats)
+            torch.cuda.synchronize()
+            assert gix.last_status() & 32, with_stats
+            # ... and the index answers normally afterwards
+            got = _gpu_search(libs, gix, wl.queries, wl.lo, wl.hi, 10, 32, budget=64)
+            _assert_parity(got, ref)
+            assert gix.last_status() == 0
+    finally:
+        gix.close()
+
+
 @pytest.mark.parametrize("name,n,nq", [("sift", 60_000, 300), ("deep1m", 50_000, 300), ("deep10m", 70_001, 300)])
 def test_visited_hash_table_form(libs, cache_dir, name, n, nq):
     """The visited set as a hash table of ranks in global scratch (what large indexes get at beam widths
