@@ -344,17 +344,19 @@ def sweep_operating_point(frog, torch, b: Batch, budgets, beams, tag=""):
         for ef in beams:
             if ef < k:
                 continue
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
             b.search(ef, prm)   # warm
-            e0.record()
-            b.search(ef, prm)
-            e1.record()
+            evs[0].record()
+            for i in range(3):  # the median of three launches ranks the candidates
+                b.search(ef, prm)
+                evs[i + 1].record()
             torch.cuda.synchronize()
+            ms = sorted(evs[i].elapsed_time(evs[i + 1]) for i in range(3))[1]
             ids = b.out_ids.cpu().numpy()
             rec = recall_at_k(ids, b.gt_ids)
             rec_t = recall_tie_aware(b.out_d.cpu().numpy(), b.gt_d)
             row = {"budget": B, "beam_width": ef, "recall": round(rec, 4), "recall_tie_aware": round(rec_t, 4),
-                   "qps": round(b.wl.nq / (e0.elapsed_time(e1) * 1e-3))}
+                   "qps": round(b.wl.nq / (ms * 1e-3))}
             rows.append(row)
             log(f"[bench]{tag} B={B} ef_s={ef}: recall@{k}={rec:.4f} (tie-aware {rec_t:.4f}) {row['qps']} q/s")
             if rec >= RECALL_TARGET or len(beams) == 1:
